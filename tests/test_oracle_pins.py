@@ -1,0 +1,334 @@
+"""Pins of the CPU oracle against things other than itself (no GPU needed).
+
+Each test fixes the oracle to what the paper's definitions and plain mathematics determine:
+hand cases, brute force over a small alphabet, invariants, closed forms, and special cases that
+reduce to a library routine (numpy / torch matmul in fp64).
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_26632_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16_bits(vals):
+    """Exact conversion of floats that are representable in bf16 to their bit patterns."""
+    t = torch.tensor(vals, dtype=torch.float32)
+    b = t.to(torch.bfloat16)
+    assert torch.equal(b.to(torch.float32), t) or torch.isnan(t).any()
+    return inputs.as_u16(b)
+
+
+def tile_group(group_bits, reps=4):
+    """A [1, 16] row made of one group repeated (K must be a multiple of 16)."""
+    return np.tile(np.asarray(group_bits, dtype=np.uint16), reps)[None, :]
+
+
+# ---------------------------------------------------------------- selection ------------------
+
+def test_hand_cases_from_golden_file():
+    n = 0
+    with open(os.path.join(GOLDEN, "topk24_hand_cases.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            lhs, rhs = line.split("->")
+            x = [float(v) for v in lhs.split()]
+            i0, i1 = (int(v) for v in rhs.split())
+            X = tile_group(bf16_bits(x))
+            mask = oracle.topk24_mask(X)[0, :4]
+            want = np.zeros(4, dtype=np.uint8)
+            want[[i0, i1]] = 1
+            assert (mask == want).all(), (x, mask, want)
+            values, meta = oracle.compress(X)
+            assert (meta[0, 0] & 0xF) == (i0 | (i1 << 2))
+            assert values[0, 0] == X[0, i0] and values[0, 1] == X[0, i1]
+            n += 1
+    assert n >= 10
+
+
+def _brute_force_pair(mags):
+    """Independent definition: among the 6 index pairs, the valid ones keep magnitudes that are
+    all >= every dropped magnitude; the answer is the lexicographically smallest valid pair."""
+    best = None
+    for pair in itertools.combinations(range(4), 2):
+        dropped = [i for i in range(4) if i not in pair]
+        if min(mags[i] for i in pair) >= max(mags[i] for i in dropped):
+            if best is None or pair < best:
+                best = pair
+    return best
+
+
+def test_brute_force_small_alphabet_exhaustive():
+    # +0, -0, +-1, +-2, +-Inf, NaN, smallest subnormal, and a value with low mantissa bits
+    alphabet = np.array([0x0000, 0x8000, 0x3F80, 0xBF80, 0x4000, 0xC000, 0x7F80, 0xFF80, 0x7FC0,
+                         0x0001, 0x8001, 0x3F81], dtype=np.uint16)
+    groups = np.array(list(itertools.product(alphabet, repeat=4)), dtype=np.uint16)  # 20736 x 4
+    pad = (-len(groups)) % 4
+    groups = np.concatenate([groups, np.zeros((pad, 4), dtype=np.uint16)])
+    X = groups.reshape(-1, 16)  # 4 groups per row
+    mask = oracle.topk24_mask(X).reshape(-1, 4)
+    values, meta = oracle.compress(X)
+    nibbles = np.stack([(meta[:, 0] >> (4 * j)) & 0xF for j in range(4)], axis=1).reshape(-1)
+    for gi, grp in enumerate(groups):
+        mags = [int(b) & 0x7FFF for b in grp]
+        i0, i1 = _brute_force_pair(mags)
+        assert mask[gi].sum() == 2
+        assert mask[gi][i0] == 1 and mask[gi][i1] == 1, (grp, mask[gi], (i0, i1))
+        assert nibbles[gi] == (i0 | (i1 << 2))
+
+
+def test_selection_invariants_random():
+    rng = np.random.default_rng(7)
+    X = rng.integers(0, 1 << 16, size=(64, 256), dtype=np.uint16)  # every bit pattern class
+    mask = oracle.topk24_mask(X)
+    g = mask.reshape(64, -1, 4)
+    assert (g.sum(-1) == 2).all()
+    mag = (X & 0x7FFF).astype(np.int64).reshape(64, -1, 4)
+    kept_min = np.where(g == 1, mag, 1 << 20).min(-1)
+    drop_max = np.where(g == 0, mag, -1).max(-1)
+    assert (kept_min >= drop_max).all()
+
+
+def test_tie_goes_to_lower_index_everywhere():
+    X = np.full((1, 64), 0x3F80, dtype=np.uint16)
+    mask = oracle.topk24_mask(X)
+    assert (mask.reshape(-1, 4) == np.array([1, 1, 0, 0])).all()
+    # sign does not matter for ties
+    X[0, 1::2] = 0xBF80
+    assert (oracle.topk24_mask(X).reshape(-1, 4) == np.array([1, 1, 0, 0])).all()
+
+
+# ---------------------------------------------------------------- compression ----------------
+
+LEGAL_NIBBLES = {0x4, 0x8, 0x9, 0xC, 0xD, 0xE}
+
+
+@pytest.mark.parametrize("dist", ["gelu", "outlier", "gelu_chan"])
+def test_compress_decompress_roundtrip(dist):
+    X = inputs.as_u16(inputs.make_x(96, 256, dist, 11))
+    mask = oracle.topk24_mask(X)
+    values, meta = oracle.compress(X)
+    back = oracle.decompress(values, meta)
+    assert (back == X * mask).all()  # bit-for-bit, incl. sign of kept zeros
+    nibs = np.stack([(meta >> (4 * j)) & 0xF for j in range(4)], axis=-1).reshape(-1)
+    assert set(np.unique(nibs).tolist()) <= LEGAL_NIBBLES
+    # values are exactly the kept entries, in ascending position
+    kept = X[mask.astype(bool)].reshape(96, 128)
+    assert (kept == values).all()
+
+
+def test_exactly_two_kept_positions_even_when_values_are_zero():
+    X = np.zeros((4, 64), dtype=np.uint16)
+    X[0, 5] = 0x4000
+    mask = oracle.topk24_mask(X)
+    assert (mask.reshape(4, -1, 4).sum(-1) == 2).all()
+    values, meta = oracle.compress(X)
+    assert (oracle.decompress(values, meta) == X).all()
+
+
+def _hw_offset_independent(m, k, K):
+    """Bit address of logical element (m, k) restated from the tensor-memory picture:
+    lane-major 16-byte rows; returns (byte offset, bit in byte)."""
+    rb, r = divmod(m, 128)
+    kb, kk = divmod(k, 128)
+    col, k32 = divmod(kk, 32)           # tensor-memory column = K step
+    lane = (r % 8) + 8 * (k32 // 16) + 16 * (r // 16)
+    bit = (k32 % 16) + 16 * ((r // 8) % 2)
+    byte = (rb * (K // 128) + kb) * 2048 + lane * 16 + col * 4 + bit // 8
+    return byte, bit % 8
+
+
+def test_metadata_hw_permutation_is_bijection_and_matches_layout():
+    M, K = 200, 384  # ragged row block
+    rng = np.random.default_rng(3)
+    X = rng.integers(0, 1 << 16, size=(M, K), dtype=np.uint16)
+    _, meta = oracle.compress(X)
+    hw = oracle.meta_canon_to_hw(meta, M, K)
+    assert hw.size == 2 * 3 * 2048 == oracle.meta_hw_bytes(M, K)
+    assert (oracle.meta_hw_to_canon(hw, M, K) == meta).all()
+    # every logical element's metadata bit sits where the layout statement says
+    for m in [0, 1, 7, 8, 15, 16, 127, 128, 199]:
+        for k in [0, 3, 4, 15, 16, 31, 32, 127, 128, 383]:
+            canon_bit = (int(meta[m, k // 16]) >> (k % 16)) & 1
+            byte, bit = _hw_offset_independent(m, k, K)
+            assert ((int(hw[byte]) >> bit) & 1) == canon_bit
+    # pad rows hold the legal pattern (positions 0 and 1)
+    byte, _ = _hw_offset_independent(255, 0, K)
+    assert hw[byte] == 0x44
+    # a permutation: each hw byte written exactly once
+    marks = oracle.meta_canon_to_hw(np.full((256, K // 16), 0xFFFF, dtype=np.uint16), 256, K)
+    assert (marks == 0xFF).all()
+
+
+# ---------------------------------------------------------------- scale ----------------------
+
+def test_scale_closed_forms():
+    # every group [a,a,a,a]: dense norm^2 = 4a^2 G, kept norm^2 = 2a^2 G  ->  s = sqrt(2)
+    X = tile_group(bf16_bits([3.0, 3.0, 3.0, 3.0]), reps=16)
+    s = oracle.row_scale(X, oracle.COMP_ROW)
+    assert abs(s[0] - np.sqrt(2.0)) < 1e-6
+    # groups [1,2,2,1]: 10 / 8
+    X = tile_group(bf16_bits([1.0, 2.0, 2.0, 1.0]), reps=8)
+    assert abs(oracle.row_scale(X, oracle.COMP_ROW)[0] - np.sqrt(1.25)) < 1e-6
+    # already 2:4 sparse rows: s = 1 up to eps
+    X = tile_group(bf16_bits([0.0, -5.0, 0.0, 0.25]), reps=8)
+    assert abs(oracle.row_scale(X, oracle.COMP_ROW)[0] - 1.0) < 1e-7
+    # all-zero row: s = 0 (no NaN)
+    X = np.zeros((1, 32), dtype=np.uint16)
+    assert oracle.row_scale(X, oracle.COMP_ROW)[0] == 0.0
+    # mode none
+    assert (oracle.row_scale(X, oracle.COMP_NONE) == 1.0).all()
+
+
+def test_scale_invariant_and_modes():
+    Xt = inputs.make_x(32, 512, "gelu", 5)
+    X = inputs.as_u16(Xt)
+    mask = oracle.topk24_mask(X).astype(np.float64)
+    xf = Xt.to(torch.float64).numpy()
+    num = (xf ** 2).sum(1)
+    den = ((xf * mask) ** 2).sum(1)
+    s = oracle.row_scale(X, oracle.COMP_ROW).astype(np.float64)
+    # s^2 (den + eps) = num
+    np.testing.assert_allclose(s ** 2 * (den + 1e-8), num, rtol=3e-7)
+    # rescaled sparse row has the dense row's norm (the stated purpose of the compensation)
+    np.testing.assert_allclose(np.sqrt(((s[:, None] * xf * mask) ** 2).sum(1)), np.sqrt(num),
+                               rtol=1e-6)
+    assert (s >= 1.0).all()
+    st = oracle.row_scale(X, oracle.COMP_TENSOR).astype(np.float64)
+    assert (st == st[0]).all()
+    np.testing.assert_allclose(st[0] ** 2 * (den.sum() + 1e-8), num.sum(), rtol=3e-7)
+
+
+# ---------------------------------------------------------------- product + epilogue ---------
+
+def test_sparse_path_equals_masked_dense_path_bitwise():
+    wl = inputs.Workload("t", 24, 256, 40, "outlier", 21)
+    d = inputs.make_workload(wl)
+    X, W = inputs.as_u16(d["X"]), inputs.as_u16(d["W"])
+    values, meta = oracle.compress(X)
+    xm = oracle.decompress(values, meta)
+    a = oracle.gemm_masked_f32(xm, W)
+    b = oracle.gemm_sparse_f32(values, meta, W)
+    assert (a.view(np.uint32) == b.view(np.uint32)).all()
+    rows = np.array([3, 0, 23], dtype=np.int64)
+    assert (oracle.gemm_sparse_f32(values, meta, W, rows) == b[rows]).all()
+
+
+def test_gemm_matches_fp64_library_matmul():
+    wl = inputs.Workload("t", 16, 512, 48, "gelu", 22)  # N != K catches a transposed W
+    d = inputs.make_workload(wl)
+    X, W = inputs.as_u16(d["X"]), inputs.as_u16(d["W"])
+    mask = torch.from_numpy(oracle.topk24_mask(X).astype(np.float64))
+    ref = (d["X"].to(torch.float64) * mask) @ d["W"].to(torch.float64).T
+    values, meta = oracle.compress(X)
+    xm = oracle.decompress(values, meta)
+    got32 = oracle.gemm_masked_f32(xm, W)
+    got64 = oracle.gemm_masked_f64(xm, W)
+    np.testing.assert_allclose(got64, ref.numpy(), rtol=1e-12, atol=1e-14)
+    err = np.linalg.norm(got32 - ref.numpy()) / np.linalg.norm(ref.numpy())
+    assert err < 1e-5  # far below the 5e-3 gate applied to the GPU result
+
+
+def test_already_sparse_input_reduces_to_dense_linear():
+    """If X is already 2:4 sparse the whole path is an ordinary linear layer."""
+    g = torch.Generator().manual_seed(5)
+    M, K, N = 20, 128, 24
+    x = torch.randn(M, K, generator=g)
+    keep = torch.zeros(M, K // 4, 4)
+    for pair_id, pair in enumerate(itertools.combinations(range(4), 2)):
+        sel = (torch.arange(M * (K // 4)).reshape(M, K // 4) % 6) == pair_id
+        for p in pair:
+            keep[..., p] += sel
+    keep = keep.reshape(M, K) > 0
+    x = torch.where(keep, x + 0.5 * torch.sign(x), torch.zeros(())).to(torch.bfloat16)
+    w = inputs.make_w(N, K, 9)
+    b = inputs.make_bias(N, 9)
+    out = oracle.act_sparse_linear(inputs.as_u16(x), inputs.as_u16(w), bias=inputs.as_u16(b),
+                                   comp_mode=oracle.COMP_ROW)
+    ref = torch.nn.functional.linear(x.double(), w.double(), b.double()).numpy()
+    np.testing.assert_allclose(out["Y"], ref, rtol=2e-5, atol=2e-6)
+    np.testing.assert_allclose(out["scale"], 1.0, atol=1e-6)
+    assert (oracle.decompress(out["values"], out["meta_canon"]) == inputs.as_u16(x)).all()
+
+
+def test_integer_valued_case_is_exact():
+    rng = np.random.default_rng(0)
+    M, K, N = 12, 64, 20
+    xi = rng.integers(-8, 9, size=(M, K))
+    wi = rng.integers(-4, 5, size=(N, K))
+    X = bf16_bits(xi.astype(np.float32).tolist())
+    W = bf16_bits(wi.astype(np.float32).tolist())
+    mask = oracle.topk24_mask(X).astype(np.int64)
+    want = (xi * mask) @ wi.T
+    values, meta = oracle.compress(X)
+    got = oracle.gemm_sparse_f32(values, meta, W)
+    assert (got == want.astype(np.float32)).all()
+
+
+def test_epilogue_closed_form_and_order():
+    acc = np.array([[1.0, -2.0]], dtype=np.float32)
+    s = np.array([2.0], dtype=np.float32)
+    bias = bf16_bits([0.5, 0.25])
+    yr = bf16_bits([[0.25, -1.0]])
+    y = oracle.epilogue(acc, 1, s=s, bias=bias, Yr=yr)
+    assert y.tolist() == [[2.75, -4.75]]  # s*acc + bias + Yr; bias and Yr are NOT scaled
+    assert oracle.epilogue(acc, 1).tolist() == [[1.0, -2.0]]
+    assert oracle.epilogue(acc, 1, bias=bias).tolist() == [[1.5, -1.75]]
+
+
+def test_whole_path_composition_and_row_subset():
+    wl = inputs.WORKLOADS["tiny"]
+    d = inputs.make_workload(wl, with_bias=True, with_residual=True, M=32)
+    X, W = inputs.as_u16(d["X"]), inputs.as_u16(d["W"])
+    bias, yr = inputs.as_u16(d["bias"]), inputs.as_u16(d["residual"])
+    full = oracle.act_sparse_linear(X, W, bias=bias, comp_mode=oracle.COMP_ROW, Yr=yr)
+    mask = oracle.topk24_mask(X).astype(np.float64)
+    xf = d["X"].double().numpy()
+    s = np.sqrt((xf ** 2).sum(1) / (((xf * mask) ** 2).sum(1) + 1e-8))
+    ref = s[:, None] * ((xf * mask) @ d["W"].double().numpy().T) + d["bias"].double().numpy() \
+        + d["residual"].double().numpy()
+    np.testing.assert_allclose(full["Y"], ref, rtol=3e-5, atol=3e-6)
+    rows = np.array([31, 2, 17], dtype=np.int64)
+    part = oracle.act_sparse_linear(X, W, bias=bias, comp_mode=oracle.COMP_ROW, Yr=yr, rows=rows)
+    assert (part["Y"] == full["Y"][rows]).all()
+
+
+def test_pruning_error_is_smaller_on_gelu_shaped_rows_than_on_gaussian_rows():
+    """Qualitative claim of the motivation section: near-zero-concentrated activations lose
+    little under 2:4 pruning.  Sanity only."""
+    def rfe(dist):
+        x = inputs.make_x(64, 512, dist, 1)
+        w = inputs.make_w(64, 512, 1)
+        X = inputs.as_u16(x)
+        mask = torch.from_numpy(oracle.topk24_mask(X).astype(np.float64))
+        full = x.double() @ w.double().T
+        sp = (x.double() * mask) @ w.double().T
+        return float((full - sp).norm() / full.norm())
+    assert rfe("gelu") < 0.6 * rfe("normal")
+
+
+def test_lora_residual_matches_library_matmul():
+    g = torch.Generator().manual_seed(2)
+    M, K, R, N = 8, 64, 16, 12
+    x = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    lb = (torch.randn(R, K, generator=g) * 0.1).to(torch.bfloat16)
+    la = (torch.randn(N, R, generator=g) * 0.1).to(torch.bfloat16)
+    got = oracle.lora_residual(inputs.as_u16(x), inputs.as_u16(lb), inputs.as_u16(la))
+    ref = (x.double() @ lb.double().T) @ la.double().T
+    np.testing.assert_allclose(got, ref.numpy(), rtol=1e-5, atol=1e-6)
+
+
+def test_bf16_rounding_routine_matches_torch():
+    g = torch.Generator().manual_seed(3)
+    v = torch.randn(4096, generator=g) * 10
+    v[:4] = torch.tensor([0.0, -0.0, float("inf"), 1.00390625])  # last one is a tie case
+    got = oracle.f32_to_bf16(v.numpy())
+    assert (got == inputs.as_u16(v.to(torch.bfloat16))).all()
