@@ -1,0 +1,171 @@
+/*
+ * lynx.h -- C ABI of the B200 (sm_100a) 2:4 activation-sparse linear layer.
+ *
+ * The library computes the hot path of RT-Lynx (Algorithm 1; Algorithm 2, activation_sparse
+ * branch): each token row of X is pruned along K to 2:4 sparsity by Top-2-of-4 magnitude,
+ * compressed to (values, 2-bit index metadata), multiplied by dense bf16 weights on the sparse
+ * tensor cores, and finished by an epilogue that applies the norm-compensation scale, the bias
+ * and an optional residual (the low-rank branch output Y_r) before one cast to bf16.
+ *
+ * General rules for every entry point
+ *   - Pointers are DEVICE pointers unless the argument is documented as HOST.
+ *   - The caller owns every buffer it passes; the library never frees or resizes them and never
+ *     modifies inputs.  Scratch memory belongs to the context (lynx_ctx).
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and returns without synchronising, except the *_host entry point which synchronises the
+ *     stream before returning.
+ *   - Errors are return values; nothing throws and nothing aborts.  Argument errors are found on
+ *     the host before any launch.  A device-side wait that ran out (should never happen) is
+ *     reported as LYNX_ERR_TIMEOUT by the next call on the same context or by lynx_last_error.
+ *   - Layouts: X is M x K bf16 row-major with leading dimension ldx (elements); W is N x K bf16
+ *     row-major (a Linear weight, D_out x D_in) with leading dimension ldw; Y is M x N bf16
+ *     row-major with leading dimension ldy; bias is N bf16; residual is M x N bf16, ld = ldr.
+ *   - Shape rules: M >= 1, K % 128 == 0, N % 8 == 0; base pointers and leading dimensions must be
+ *     16-byte aligned (ld % 8 == 0 for bf16).  Row tails (M not a multiple of the tile) are
+ *     handled inside the kernels.
+ *   - There is no CPU fallback: on a device that is not sm_100 lynx_create fails with
+ *     LYNX_ERR_UNSUPPORTED_ARCH.
+ */
+#ifndef LYNX_H_
+#define LYNX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define LYNX_API __attribute__((visibility("default")))
+#else
+#define LYNX_API
+#endif
+
+typedef struct lynx_ctx lynx_ctx; /* opaque: scratch workspace, descriptor cache, error word */
+
+typedef enum {
+    LYNX_OK = 0,
+    LYNX_ERR_INVALID_ARG = 1,
+    LYNX_ERR_UNSUPPORTED_SHAPE = 2,
+    LYNX_ERR_ALIGNMENT = 3,
+    LYNX_ERR_WORKSPACE = 4,
+    LYNX_ERR_CUDA = 5,
+    LYNX_ERR_TIMEOUT = 6,
+    LYNX_ERR_UNSUPPORTED_ARCH = 7
+} lynx_status;
+
+/* Norm compensation of Algorithm 1 line 4:  s = sqrt(||X||^2 / (||X~||^2 + 1e-8)). */
+typedef enum {
+    LYNX_COMP_NONE = 0,  /* no rescaling: y = x~ W^T + b  (Algorithm 2, activation_sparse)   */
+    LYNX_COMP_ROW = 1,   /* one s per token row (the reading used by default)                */
+    LYNX_COMP_TENSOR = 2 /* one s for the whole X (Algorithm 1 read literally)               */
+} lynx_comp_mode;
+
+typedef enum {
+    LYNX_FUSE_AUTO = 0,     /* library picks                                                  */
+    LYNX_FUSE_SEPARATE = 1, /* prune/compress kernel, then sparse GEMM kernel                 */
+    LYNX_FUSE_FUSED = 2     /* one kernel, compressed activations never written to HBM        */
+} lynx_fuse_mode;
+
+/* Epilogue terms of lynx_sparse_linear (all optional). */
+typedef struct {
+    const float* row_scale; /* [M] fp32 per-row scale s_m, or NULL (= 1)                      */
+    const void* residual;   /* Y_r: [M x N] bf16, leading dimension ldr, or NULL              */
+    int64_t ldr;
+} lynx_comp;
+
+/* ---- context ------------------------------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device` (made current for the call).  Allocates a small
+ * status word; scratch is allocated lazily (see lynx_reserve).  */
+LYNX_API lynx_status lynx_create(lynx_ctx** out, int device);
+/* Frees the context's scratch.  The caller must have synchronised every stream it used. */
+LYNX_API lynx_status lynx_destroy(lynx_ctx* ctx);
+LYNX_API const char* lynx_status_string(lynx_status s);
+/* Reads and clears the sticky device-side error word (LYNX_OK or LYNX_ERR_TIMEOUT). HOST call,
+ * does not synchronise: call after synchronising the stream to be sure a launch has finished. */
+LYNX_API lynx_status lynx_last_error(lynx_ctx* ctx);
+
+/* Bytes of the compressed operands for an M x K activation matrix. */
+LYNX_API size_t lynx_values_bytes(int64_t M, int64_t K); /* M * (K/2) bf16                    */
+LYNX_API size_t lynx_meta_bytes(int64_t M, int64_t K);   /* ceil(M/128) * (K/128) * 2048      */
+/* Scratch the context needs for lynx_act_sparse_linear / TENSOR compensation at this size. */
+LYNX_API size_t lynx_workspace_bytes(int64_t M, int64_t N, int64_t K);
+/* Grows the context's scratch to serve shapes up to (M, N, K).  May call cudaMalloc and
+ * synchronise; call it outside timed or captured regions.  Entry points that need scratch call
+ * it themselves when the scratch is too small. */
+LYNX_API lynx_status lynx_reserve(lynx_ctx* ctx, int64_t M, int64_t N, int64_t K);
+
+/* ---- step 1-4: Top-2-of-4 selection, compression, norm-compensation scale --------------------
+ * (Algorithm 1 lines 3-4; sparse-tensor-core appendix for the values + 2-bit index form.)
+ *
+ * For every row m and group g of 4 consecutive elements (groups start at k = 0) keeps the two
+ * elements of largest magnitude; magnitudes compare as the 15 non-sign bits of the bf16 pattern
+ * (so NaN > Inf > finite, +0 == -0, no flush of subnormals) and ties go to the lower index.
+ *   values[m, 2g+j] = X[m, 4g + idx_j], idx_0 < idx_1          (bit copies)   [M x K/2 bf16]
+ *   meta: nibble(m, g) = idx_0 | idx_1 << 2, stored in the order the sparse MMA reads it:
+ *         blocks of 128 rows x 128 K-elements, 2048 bytes each, block (rb, kb) at byte
+ *         (rb * K/128 + kb) * 2048; inside a block, byte = lane*16 + step*4 + ((r/8)%2)*2 + h/8
+ *         with r = row in block, step = (k%128)/32, lane = r%8 + 8*((k%32)/16) + 16*(r/16),
+ *         h = k%16 (bit h%8 of that byte belongs to element k).  Rows past M in the last block
+ *         are filled with the pattern 0x4.  lynx_meta_to_canonical converts to the plain
+ *         row-major form for inspection.
+ *   row_scale (may be NULL when mode == LYNX_COMP_NONE): [M] fp32, s_m per `mode`
+ *         (ROW: per row; TENSOR: the same global s in every entry; NONE: 1.0 if non-NULL).
+ * TENSOR mode uses the context's scratch (2 floats per row).
+ */
+LYNX_API lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
+                                         int64_t ldx, void* values, void* meta, float* row_scale,
+                                         lynx_comp_mode mode, void* stream);
+
+/* ---- step 5-6: 2:4 sparse x dense product and epilogue ---------------------------------------
+ * (Algorithm 1 lines 5-6; Algorithm 2 for the bias.)
+ *   Y[m, n] = bf16_rne( s_m * sum_k X~[m,k] W[n,k]  +  bias[n]  +  Y_r[m,n] )
+ * where X~ is the matrix (values, meta) encodes, the sum is accumulated in fp32 on the sparse
+ * tensor cores, and absent terms (bias == NULL, comp == NULL or its members NULL) are 1 / 0.
+ * values / meta must have the layout lynx_prune_compress writes.
+ */
+LYNX_API lynx_status lynx_sparse_linear(lynx_ctx* ctx, const void* values, const void* meta,
+                                        int64_t M, int64_t K, const void* W, int64_t N, int64_t ldw,
+                                        const void* bias, const lynx_comp* comp, void* Y,
+                                        int64_t ldy, void* stream);
+
+/* ---- whole layer (Algorithm 1) -----------------------------------------------------------------
+ * Y = act_sparse_linear(X, W, bias, residual) = steps 1-6 above.  SEPARATE runs the two kernels
+ * back to back on `stream` with the compressed operands in the context's scratch (grown on
+ * demand: see lynx_reserve); FUSED prunes inside the GEMM kernel.  Both give the same values,
+ * metadata and (up to fp32 summation order) the same Y.
+ */
+LYNX_API lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
+                                            int64_t ldx, const void* W, int64_t N, int64_t ldw,
+                                            const void* bias, lynx_comp_mode mode,
+                                            const void* residual, int64_t ldr, void* Y, int64_t ldy,
+                                            lynx_fuse_mode fuse, void* stream);
+
+/* Same layer with the activations and the result in HOST memory (pinned memory recommended):
+ * X_host [M x K] and Y_host [M x N] are dense row-major bf16 HOST buffers; W and bias stay
+ * DEVICE resident (weights are loaded once).  Copies X to the device, runs the layer, copies Y
+ * back and synchronises `stream`.  Staging buffers live in the context's scratch. */
+LYNX_API lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_host, int64_t M,
+                                                 int64_t K, const void* W, int64_t N, int64_t ldw,
+                                                 const void* bias, lynx_comp_mode mode, void* Y_host,
+                                                 lynx_fuse_mode fuse, void* stream);
+
+/* ---- inspection helpers ------------------------------------------------------------------------ */
+
+/* Hardware-order metadata -> canonical form: uint16 [M x K/16], nibble (g%4) of group g in bits
+ * 4*(g%4).. of word g/4 of its row. */
+LYNX_API lynx_status lynx_meta_to_canonical(lynx_ctx* ctx, const void* meta, int64_t M, int64_t K,
+                                            void* meta_canon, void* stream);
+/* Expands (values, meta) back to the masked dense matrix X~ [M x K] bf16 (dropped entries +0). */
+LYNX_API lynx_status lynx_decompress(lynx_ctx* ctx, const void* values, const void* meta, int64_t M,
+                                     int64_t K, void* Xmasked, void* stream);
+
+/* Number of kernels the library launched on this context since creation (for accounting). */
+LYNX_API int64_t lynx_launch_count(lynx_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LYNX_H_ */

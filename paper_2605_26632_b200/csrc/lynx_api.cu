@@ -1,0 +1,394 @@
+// C ABI of the library (see include/lynx.h): argument checks, context (scratch, error word,
+// launch counter), TMA descriptor construction and kernel launches.  No CPU fallback anywhere.
+#include "../../include/lynx.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "prune_compress.cuh"
+#include "sparse_gemm.cuh"
+
+using namespace lynx;
+
+struct lynx_ctx {
+    int device = 0;
+    int num_sms = 0;
+    uint32_t* err_host = nullptr;  // mapped pinned word written by kernels
+    uint32_t* err_dev = nullptr;
+    void* scratch = nullptr;  // compressed operands, scale, sums, host staging mirrors
+    size_t scratch_bytes = 0;
+    int64_t launches = 0;
+    int gemm_cfg = 0;  // 0 = auto
+    std::mutex mu;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// 2D row-major tensor [rows x cols] of `elem_bytes` elements, row pitch `ld_bytes`.
+bool make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t rows,
+                  uint64_t cols, uint64_t ld_bytes, uint32_t box_cols, uint32_t box_rows,
+                  CUtensorMapSwizzle sw) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ld_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    (void)elem_bytes;
+    return enc(m, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+lynx_status check_device_error(lynx_ctx* ctx) {
+    if (ctx->err_host && *ctx->err_host != DEV_OK) return LYNX_ERR_TIMEOUT;
+    return LYNX_OK;
+}
+
+lynx_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? LYNX_OK : LYNX_ERR_CUDA; }
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Scratch layout for (M, N, K): [values][meta][row_scale M floats][sums 2M floats][X stage][Y stage]
+struct ScratchLayout {
+    size_t values, meta, scale, sums, xstage, ystage, total;
+};
+ScratchLayout scratch_layout(int64_t M, int64_t N, int64_t K) {
+    ScratchLayout L;
+    size_t off = 0;
+    L.values = off; off = align_up(off + lynx_values_bytes(M, K), 1024);
+    L.meta = off;   off = align_up(off + lynx_meta_bytes(M, K), 1024);
+    L.scale = off;  off = align_up(off + (size_t)M * 4, 1024);
+    L.sums = off;   off = align_up(off + (size_t)M * 8, 1024);
+    L.xstage = off; off = align_up(off + (size_t)M * K * 2, 1024);
+    L.ystage = off; off = align_up(off + (size_t)M * N * 2, 1024);
+    L.total = off;
+    return L;
+}
+
+// --------------------------------------------------------------------------- GEMM launch -----
+
+template <class Cfg>
+lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
+                            const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
+                            void* Y, int64_t ldy, cudaStream_t st) {
+    CUtensorMap ta, tb, te, ty;
+    const uint64_t rb = (uint64_t)((M + 127) / 128), kblocks = (uint64_t)(K / 128);
+    if (!make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, values, (uint64_t)M, (uint64_t)(K / 2),
+                      (uint64_t)K, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)N, (uint64_t)K, (uint64_t)ldw * 2, 64,
+                      Cfg::BN_CTA, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&te, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, meta, rb * kblocks * 2, 256, 1024, 256, 2,
+                      CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, 64,
+                      32, CU_TENSOR_MAP_SWIZZLE_128B))
+        return LYNX_ERR_CUDA;
+
+    GemmParams p;
+    p.M = M; p.N = N; p.K = K;
+    p.row_scale = comp ? comp->row_scale : nullptr;
+    p.bias = static_cast<const uint16_t*>(bias);
+    p.residual = comp ? static_cast<const uint16_t*>(comp->residual) : nullptr;
+    p.ldr = comp ? comp->ldr : 0;
+    p.dev_error = ctx->err_dev;
+    p.tiles_m = (int)((M + Cfg::BM * Cfg::CG - 1) / (Cfg::BM * Cfg::CG));
+    p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
+
+    auto kern = sparse_gemm_kernel<Cfg>;
+    static bool attr_set = false;  // per instantiation
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
+            return LYNX_ERR_CUDA;
+        attr_set = true;
+    }
+    const int tiles = p.tiles_m * p.tiles_n;
+    int clusters = ctx->num_sms / Cfg::CG;
+    if (clusters > tiles) clusters = tiles;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(clusters * Cfg::CG));
+    cfg.blockDim = dim3(Cfg::THREADS);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = Cfg::CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, te, ty, p);
+    if (e != cudaSuccess) return LYNX_ERR_CUDA;
+    ctx->launches++;
+    return LYNX_OK;
+}
+
+lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K, const void* W,
+                        int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp, void* Y, int64_t ldy,
+                        cudaStream_t st) {
+    int cfg = ctx->gemm_cfg;
+    if (cfg == 0) cfg = 1;
+#define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, Y, ldy, st
+    switch (cfg) {
+        case 1: return launch_gemm_cfg<GemmCfg<128, 1, 4, 1>>(LYNX_GEMM_ARGS);
+        case 2: return launch_gemm_cfg<GemmCfg<192, 1, 3, 1>>(LYNX_GEMM_ARGS);
+        case 3: return launch_gemm_cfg<GemmCfg<256, 1, 2, 1>>(LYNX_GEMM_ARGS);
+        case 4: return launch_gemm_cfg<GemmCfg<192, 2, 4, 2>>(LYNX_GEMM_ARGS);
+        case 5: return launch_gemm_cfg<GemmCfg<256, 2, 4, 1>>(LYNX_GEMM_ARGS);
+        case 6: return launch_gemm_cfg<GemmCfg<128, 2, 5, 2>>(LYNX_GEMM_ARGS);
+        default: return LYNX_ERR_INVALID_ARG;
+    }
+#undef LYNX_GEMM_ARGS
+}
+
+lynx_status check_common(lynx_ctx* ctx, int64_t M, int64_t K) {
+    if (!ctx) return LYNX_ERR_INVALID_ARG;
+    if (M < 1 || K < 128) return LYNX_ERR_INVALID_ARG;
+    if (K % 128 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    if (M > (1ll << 30) || K > (1ll << 30)) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    return LYNX_OK;
+}
+
+lynx_status ensure_scratch(lynx_ctx* ctx, size_t bytes) {
+    if (ctx->scratch_bytes >= bytes) return LYNX_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) return LYNX_ERR_CUDA;
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    ctx->scratch = nullptr;
+    ctx->scratch_bytes = 0;
+    if (cudaMalloc(&ctx->scratch, bytes) != cudaSuccess) return LYNX_ERR_WORKSPACE;
+    ctx->scratch_bytes = bytes;
+    return LYNX_OK;
+}
+
+}  // namespace
+
+// ================================================================================ C ABI ==========
+
+extern "C" {
+
+lynx_status lynx_create(lynx_ctx** out, int device) {
+    if (!out) return LYNX_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return LYNX_ERR_CUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return LYNX_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return LYNX_ERR_CUDA;
+    if (prop.major != 10) return LYNX_ERR_UNSUPPORTED_ARCH;
+    if (!get_encode()) return LYNX_ERR_CUDA;
+    lynx_ctx* ctx = new (std::nothrow) lynx_ctx();
+    if (!ctx) return LYNX_ERR_WORKSPACE;
+    ctx->device = device;
+    ctx->num_sms = prop.multiProcessorCount;
+    if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->err_host), 64, cudaHostAllocMapped) != cudaSuccess ||
+        cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->err_dev), ctx->err_host, 0) != cudaSuccess) {
+        delete ctx;
+        return LYNX_ERR_CUDA;
+    }
+    *ctx->err_host = DEV_OK;
+    const char* env = getenv("LYNX_GEMM_CFG");  // development override of the tile configuration
+    if (env) ctx->gemm_cfg = atoi(env);
+    *out = ctx;
+    return LYNX_OK;
+}
+
+lynx_status lynx_destroy(lynx_ctx* ctx) {
+    if (!ctx) return LYNX_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->err_host) cudaFreeHost(ctx->err_host);
+    delete ctx;
+    return LYNX_OK;
+}
+
+const char* lynx_status_string(lynx_status s) {
+    switch (s) {
+        case LYNX_OK: return "ok";
+        case LYNX_ERR_INVALID_ARG: return "invalid argument";
+        case LYNX_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (need K % 128 == 0, N % 8 == 0)";
+        case LYNX_ERR_ALIGNMENT: return "pointer or leading dimension not 16-byte aligned";
+        case LYNX_ERR_WORKSPACE: return "scratch allocation failed";
+        case LYNX_ERR_CUDA: return "CUDA runtime error";
+        case LYNX_ERR_TIMEOUT: return "device-side wait timed out";
+        case LYNX_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+    }
+    return "unknown status";
+}
+
+lynx_status lynx_last_error(lynx_ctx* ctx) {
+    if (!ctx) return LYNX_ERR_INVALID_ARG;
+    lynx_status s = check_device_error(ctx);
+    *ctx->err_host = DEV_OK;
+    return s;
+}
+
+size_t lynx_values_bytes(int64_t M, int64_t K) { return (size_t)M * (size_t)(K / 2) * 2; }
+size_t lynx_meta_bytes(int64_t M, int64_t K) { return (size_t)((M + 127) / 128) * (size_t)(K / 128) * 2048; }
+size_t lynx_workspace_bytes(int64_t M, int64_t N, int64_t K) { return scratch_layout(M, N, K).total; }
+
+lynx_status lynx_reserve(lynx_ctx* ctx, int64_t M, int64_t N, int64_t K) {
+    if (!ctx || M < 1 || N < 1 || K < 1) return LYNX_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    return ensure_scratch(ctx, scratch_layout(M, N, K).total);
+}
+
+int64_t lynx_launch_count(lynx_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, void* values,
+                                void* meta, float* row_scale, lynx_comp_mode mode, void* stream) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if (!X || !values || !meta) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW && mode != LYNX_COMP_TENSOR) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_NONE && !row_scale) return LYNX_ERR_INVALID_ARG;
+    if (ldx < K) return LYNX_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(values) || !aligned16(meta) || (ldx % 16) != 0 ||
+        (reinterpret_cast<uintptr_t>(X) & 31u) || (reinterpret_cast<uintptr_t>(values) & 31u))
+        return LYNX_ERR_ALIGNMENT;  // 32-byte vector accesses
+    if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* sums = nullptr;
+    if (mode == LYNX_COMP_TENSOR) {
+        std::lock_guard<std::mutex> lock(ctx->mu);
+        ScratchLayout L = scratch_layout(M, 8, K);
+        if (ctx->scratch_bytes < L.sums + (size_t)M * 8) {
+            if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
+        }
+        sums = reinterpret_cast<float*>(static_cast<char*>(ctx->scratch) + L.sums);
+    }
+    const unsigned grid = (unsigned)(((M + 127) / 128) * (128 / PRUNE_ROWS));
+    if (mode == LYNX_COMP_NONE)
+        prune_compress_kernel<false><<<grid, PRUNE_THREADS, 0, st>>>(
+            static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
+            row_scale, nullptr, 0);
+    else
+        prune_compress_kernel<true><<<grid, PRUNE_THREADS, 0, st>>>(
+            static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
+            row_scale, sums, (int)mode);
+    ctx->launches++;
+    if (mode == LYNX_COMP_TENSOR) {
+        tensor_scale_kernel<<<1, 1024, 0, st>>>(sums, M, row_scale);
+        ctx->launches++;
+    }
+    return cuda_ok(cudaGetLastError());
+}
+
+lynx_status lynx_sparse_linear(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
+                               const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
+                               void* Y, int64_t ldy, void* stream) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if (!values || !meta || !W || !Y || N < 8) return LYNX_ERR_INVALID_ARG;
+    if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    if (ldw < K || ldy < N) return LYNX_ERR_INVALID_ARG;
+    if (!aligned16(values) || !aligned16(meta) || !aligned16(W) || !aligned16(Y) || (ldw % 8) || (ldy % 8))
+        return LYNX_ERR_ALIGNMENT;
+    if (bias && !aligned16(bias)) return LYNX_ERR_ALIGNMENT;
+    if (comp && comp->residual) {
+        if (comp->ldr < N) return LYNX_ERR_INVALID_ARG;
+        if (!aligned16(comp->residual) || (comp->ldr % 8)) return LYNX_ERR_ALIGNMENT;
+    }
+    if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+    return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, comp, Y, ldy, static_cast<cudaStream_t>(stream));
+}
+
+lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, const void* W,
+                                   int64_t N, int64_t ldw, const void* bias, lynx_comp_mode mode,
+                                   const void* residual, int64_t ldr, void* Y, int64_t ldy, lynx_fuse_mode fuse,
+                                   void* stream) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if (fuse != LYNX_FUSE_AUTO && fuse != LYNX_FUSE_SEPARATE && fuse != LYNX_FUSE_FUSED) return LYNX_ERR_INVALID_ARG;
+    if (fuse == LYNX_FUSE_FUSED) return LYNX_ERR_UNSUPPORTED_SHAPE;  // fused kernel: not built yet
+    if (N < 8) return LYNX_ERR_INVALID_ARG;
+    ScratchLayout L = scratch_layout(M, N, K);
+    {
+        std::lock_guard<std::mutex> lock(ctx->mu);
+        if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
+    }
+    char* base = static_cast<char*>(ctx->scratch);
+    void* values = base + L.values;
+    void* meta = base + L.meta;
+    float* scale = reinterpret_cast<float*>(base + L.scale);
+    s = lynx_prune_compress(ctx, X, M, K, ldx, values, meta, mode == LYNX_COMP_NONE ? nullptr : scale, mode, stream);
+    if (s != LYNX_OK) return s;
+    lynx_comp comp;
+    comp.row_scale = mode == LYNX_COMP_NONE ? nullptr : scale;
+    comp.residual = residual;
+    comp.ldr = ldr;
+    return lynx_sparse_linear(ctx, values, meta, M, K, W, N, ldw, bias, &comp, Y, ldy, stream);
+}
+
+lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_host, int64_t M, int64_t K, const void* W,
+                                        int64_t N, int64_t ldw, const void* bias, lynx_comp_mode mode, void* Y_host,
+                                        lynx_fuse_mode fuse, void* stream) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if (!X_host || !Y_host || N < 8) return LYNX_ERR_INVALID_ARG;
+    ScratchLayout L = scratch_layout(M, N, K);
+    {
+        std::lock_guard<std::mutex> lock(ctx->mu);
+        if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* base = static_cast<char*>(ctx->scratch);
+    void* xd = base + L.xstage;
+    void* yd = base + L.ystage;
+    if (cudaMemcpyAsync(xd, X_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return LYNX_ERR_CUDA;
+    s = lynx_act_sparse_linear(ctx, xd, M, K, K, W, N, ldw, bias, mode, nullptr, 0, yd, N, fuse, stream);
+    if (s != LYNX_OK) return s;
+    if (cudaMemcpyAsync(Y_host, yd, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return LYNX_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return LYNX_ERR_CUDA;
+    return check_device_error(ctx);
+}
+
+lynx_status lynx_meta_to_canonical(lynx_ctx* ctx, const void* meta, int64_t M, int64_t K, void* meta_canon,
+                                   void* stream) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if (!meta || !meta_canon) return LYNX_ERR_INVALID_ARG;
+    const int64_t n = M * (K / 16);
+    meta_to_canonical_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint8_t*>(meta), M, K, static_cast<uint16_t*>(meta_canon));
+    ctx->launches++;
+    return cuda_ok(cudaGetLastError());
+}
+
+lynx_status lynx_decompress(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
+                            void* Xmasked, void* stream) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if (!values || !meta || !Xmasked) return LYNX_ERR_INVALID_ARG;
+    const int64_t n = M * (K / 4);
+    decompress_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint16_t*>(values), static_cast<const uint8_t*>(meta), M, K, static_cast<uint16_t*>(Xmasked));
+    ctx->launches++;
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // extern "C"

@@ -1,0 +1,302 @@
+// 2:4 sparse x dense GEMM with fused epilogue for sm_100a (Algorithm 1 lines 5-6):
+//     Y[m, n] = bf16( s_m * sum_k X~[m,k] W[n,k] + bias[n] + Yr[m,n] )
+// X~ arrives compressed: values [M x K/2] bf16 and hardware-order 2-bit index metadata.
+//
+// Persistent, warp-specialised kernel.  Per CTA (or CTA pair when CG == 2):
+//   warp 0      producer: TMA loads of the compressed-A tile (128 rows x 64 stored values =
+//               128 logical K), the metadata block (2048 bytes) and the W tile into a ring of
+//               STAGES shared-memory stages guarded by full/empty mbarriers
+//   warp 1      MMA issuer (one thread): copies the stage's metadata into tensor memory
+//               (tcgen05.cp), issues four tcgen05.mma.sp kind::f16 (K = 32 logical each) into a
+//               tensor-memory fp32 accumulator, commits to the stage's empty barrier; after the
+//               last K block commits to the accumulator's full barrier
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), apply
+//               row scale / bias / residual, round to bf16, stage in swizzled shared memory and
+//               TMA-store 32 x 64 boxes
+// With two accumulator buffers the epilogue of tile i overlaps the main loop of tile i+1.
+//
+// CG == 2: the pair computes a 256 x BN tile; each CTA stages its own 128 rows of A and
+// metadata and its own BN/2 rows of W (plain TMA loads, no multicast), the leader CTA issues
+// cta_group::2 MMAs, and each CTA drains its own 128 accumulator rows.
+#pragma once
+
+#include "ptx.cuh"
+
+namespace lynx {
+
+struct GemmParams {
+    int64_t M, N, K;
+    const float* row_scale;    // [M] or nullptr
+    const uint16_t* bias;      // [N] bf16 or nullptr
+    const uint16_t* residual;  // [M x N] bf16 (ld = ldr) or nullptr
+    int64_t ldr;
+    uint32_t* dev_error;  // sticky error word (host-visible)
+    int tiles_m, tiles_n;
+};
+
+template <int BN_, int CG_, int STAGES_, int CBUFS_>
+struct GemmCfg {
+    static constexpr int BN = BN_, CG = CG_, STAGES = STAGES_, CBUFS = CBUFS_;
+    static constexpr int BM = 128;  // rows per CTA
+    static constexpr int BK = 128;  // logical K per stage
+    static constexpr int BN_CTA = BN / CG;
+    static constexpr int A_BYTES = BM * (BK / 2) * 2;     // 16 KB
+    static constexpr int B_HALF_BYTES = BN_CTA * 64 * 2;  // one 64-element K slice of the W tile
+    static constexpr int B_BYTES = 2 * B_HALF_BYTES;
+    static constexpr int E_BYTES = 2048;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
+    static constexpr int C_BOX_BYTES = 32 * 64 * 2;  // one warp's 32 x 64 bf16 store box
+    static constexpr int C_BYTES = 4 * CBUFS * C_BOX_BYTES;
+    static constexpr int ACC_STAGES = (2 * BN + 4 * STAGES <= 512) ? 2 : 1;
+    static constexpr int E_COL0 = ACC_STAGES * BN;  // metadata columns start after accumulators
+    static constexpr int TMEM_COLS = 512;
+    static constexpr int NUM_BARS = 2 * STAGES + 2 * ACC_STAGES;
+    static constexpr int SMEM_BYTES = 1024 /*align slack*/ + STAGES * STAGE_BYTES + C_BYTES + 256;
+    static constexpr int THREADS = 192;
+    static_assert(BN % (16 * CG) == 0 && BN <= 256, "tile N");
+    static_assert(BN % 64 == 0, "epilogue works on 64-column chunks");
+    static_assert(B_HALF_BYTES % 1024 == 0, "swizzle atoms need 1024-byte aligned tiles");
+    static_assert(E_COL0 % 4 == 0 && E_COL0 + 4 * STAGES <= TMEM_COLS, "tensor memory budget");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+};
+
+// Instruction descriptor of tcgen05.mma.sp kind::f16: bf16 x bf16 -> fp32, both operands
+// K-major, sparse, M x N per instruction.
+__host__ __device__ constexpr uint32_t make_idesc_sp_bf16(int m, int n) {
+    return (1u << 2)                        // sparse
+           | (1u << 4)                      // D format: fp32
+           | (1u << 7)                      // A format: bf16
+           | (1u << 10)                     // B format: bf16
+           | ((uint32_t)(n >> 3) << 17)     // N / 8
+           | ((uint32_t)(m >> 4) << 24);    // M / 16
+}
+
+template <class Cfg>
+__global__ void __launch_bounds__(Cfg::THREADS, 1)
+sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                   const __grid_constant__ CUtensorMap tmap_e, const __grid_constant__ CUtensorMap tmap_y,
+                   const GemmParams p) {
+    constexpr int CG = Cfg::CG, STAGES = Cfg::STAGES, BN = Cfg::BN;
+    extern __shared__ uint8_t smem_raw[];
+    // 1024-byte alignment for the swizzled tiles
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t sA = smem_base;
+    const uint32_t sB = sA + STAGES * Cfg::A_BYTES;
+    const uint32_t sE = sB + STAGES * Cfg::B_BYTES;
+    const uint32_t sC = sE + STAGES * Cfg::E_BYTES;
+    const uint32_t sBar = sC + Cfg::C_BYTES;
+    const uint32_t bar_full = sBar, bar_empty = sBar + 8 * STAGES;
+    const uint32_t bar_tfull = sBar + 16 * STAGES, bar_tempty = bar_tfull + 8 * Cfg::ACC_STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + (sBar - smem_base) + 8 * Cfg::NUM_BARS);
+    volatile uint32_t* cta_abort = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = (CG == 2) ? cluster_ctarank() : 0u;
+    const bool leader = rank == 0;
+    const int cluster_id = blockIdx.x / CG, num_clusters = gridDim.x / CG;
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int kblocks = (int)(p.K / Cfg::BK);
+
+    if (threadIdx.x == 0) {
+        *cta_abort = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);   // leader's producer arrives once (+ transaction bytes)
+            mbar_init(bar_empty + 8 * s, 1);  // one tcgen05.commit
+        }
+        for (int a = 0; a < Cfg::ACC_STAGES; ++a) {
+            mbar_init(bar_tfull + 8 * a, 1);         // one tcgen05.commit
+            mbar_init(bar_tempty + 8 * a, 4 * CG);   // one arrive per epilogue warp of the pair
+        }
+        fence_mbar_init();
+        prefetch_tmap(&tmap_a);
+        prefetch_tmap(&tmap_b);
+        prefetch_tmap(&tmap_e);
+        prefetch_tmap(&tmap_y);
+    }
+    if (warp == 1) {
+        tmem_alloc<CG>(smem_u32(tmem_slot), Cfg::TMEM_COLS);
+        tmem_relinquish<CG>();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if constexpr (CG == 2) cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer ----------
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0;
+            bool ok = true;
+            const uint32_t full0 = (CG == 2) ? mapa(bar_full, 0) : bar_full;  // leader's barriers
+            for (int t = cluster_id; t < num_tiles && ok; t += num_clusters) {
+                const int tm = t % p.tiles_m, tn = t / p.tiles_m;
+                const int m0 = (tm * CG + (int)rank) * Cfg::BM;
+                const int n0 = tn * BN + (int)rank * Cfg::BN_CTA;
+                const int eblk = (tm * CG + (int)rank) * kblocks;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, cta_abort, p.dev_error)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t a_dst = sA + stage * Cfg::A_BYTES;
+                    const uint32_t b_dst = sB + stage * Cfg::B_BYTES;
+                    const uint32_t e_dst = sE + stage * Cfg::E_BYTES;
+                    if constexpr (CG == 1) {
+                        const uint32_t bar = bar_full + 8 * stage;
+                        mbar_arrive_expect_tx(bar, Cfg::STAGE_BYTES);
+                        tma_load_2d(a_dst, &tmap_a, kb * 64, m0, bar);
+                        tma_load_2d(e_dst, &tmap_e, 0, 2 * (eblk + kb), bar);
+                        tma_load_2d(b_dst, &tmap_b, kb * 128, n0, bar);
+                        tma_load_2d(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * 128 + 64, n0, bar);
+                    } else {
+                        const uint32_t bar = full0 + 8 * stage;
+                        // the leader announces the bytes of both CTAs; the peer's bytes may land
+                        // first (the count goes negative for a moment, which is allowed)
+                        if (leader) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * Cfg::STAGE_BYTES);
+                        tma_load_2d_pair(a_dst, &tmap_a, kb * 64, m0, bar);
+                        tma_load_2d_pair(e_dst, &tmap_e, 0, 2 * (eblk + kb), bar);
+                        tma_load_2d_pair(b_dst, &tmap_b, kb * 128, n0, bar);
+                        tma_load_2d_pair(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * 128 + 64, n0, bar);
+                    }
+                    ++issued;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+            (void)issued;
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer --------
+        if (leader && lane == 0) {
+            constexpr uint32_t idesc = make_idesc_sp_bf16(Cfg::BM * CG, BN);
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int t = cluster_id; t < num_tiles && ok; t += num_clusters, ++it) {
+                const int acc = (Cfg::ACC_STAGES == 2) ? (it & 1) : 0;
+                const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((it >> 1) & 1) : (it & 1);
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, cta_abort, p.dev_error)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, cta_abort, p.dev_error)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t e_tmem = tmem_base + Cfg::E_COL0 + 4 * stage;
+                    tmem_cp_128x128b<CG>(e_tmem, make_desc_rows16(sE + stage * Cfg::E_BYTES));
+                    const uint64_t a_desc = make_desc_sw128(sA + stage * Cfg::A_BYTES);
+                    const uint64_t b_desc = make_desc_sw128(sB + stage * Cfg::B_BYTES);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // A: 16 stored values = 32 bytes per step; W: 32 elements = 64 bytes per
+                        // step, steps 2,3 in the second 64-element slice
+                        const uint64_t ad = a_desc + (uint64_t)(j * 2);
+                        const uint64_t bd = b_desc + (uint64_t)((j >> 1) * (Cfg::B_HALF_BYTES >> 4) + (j & 1) * 4);
+                        mma_sp_bf16<CG>(d_tmem, ad, bd, e_tmem + (j & ~1), idesc | (uint32_t)(j & 1),
+                                        (kb > 0 || j > 0) ? 1u : 0u);
+                    }
+                    if constexpr (CG == 1) tc_commit(bar_empty + 8 * stage);
+                    else tc_commit_pair(bar_empty + 8 * stage, 0x3);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                if constexpr (CG == 1) tc_commit(bar_tfull + 8 * acc);
+                else tc_commit_pair(bar_tfull + 8 * acc, 0x3);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue ----------
+        const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+        const uint32_t cbuf0 = sC + (warp - 2) * Cfg::CBUFS * Cfg::C_BOX_BYTES;
+        const uint32_t tempty0 = (CG == 2) ? mapa(bar_tempty, 0) : bar_tempty;
+        int it = 0, cb = 0;
+        for (int t = cluster_id; t < num_tiles; t += num_clusters, ++it) {
+            const int tm = t % p.tiles_m, tn = t / p.tiles_m;
+            const int acc = (Cfg::ACC_STAGES == 2) ? (it & 1) : 0;
+            const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((it >> 1) & 1) : (it & 1);
+            if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, cta_abort, p.dev_error)) break;
+            tc_fence_after();
+            const int m0 = (tm * CG + (int)rank) * Cfg::BM + q * 32;
+            const int64_t row = m0 + lane;
+            const bool row_ok = row < p.M;
+            const float s = (p.row_scale != nullptr && row_ok) ? p.row_scale[row] : 1.0f;
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 64; ++c) {
+                const int n0 = tn * BN + c * 64;
+                uint32_t v[64];
+                tmem_ld_32x32b_x32(t_row + c * 64, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                tmem_ld_32x32b_x32(t_row + c * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+                tmem_ld_wait();
+                if (c == BN / 64 - 1) {
+                    // accumulator fully read: hand it back to the MMA issuer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if constexpr (CG == 1) mbar_arrive(bar_tempty + 8 * acc);
+                        else mbar_arrive_cluster(tempty0 + 8 * acc);
+                    }
+                }
+                if (n0 >= p.N) continue;
+                // staging buffer must have been read by its previous TMA store
+                if (lane == 0) tma_store_wait_read<Cfg::CBUFS - 1>();
+                __syncwarp();
+                const uint32_t cbuf = cbuf0 + cb * Cfg::C_BOX_BYTES;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {  // 8 columns (16 bytes of output) at a time
+                    const int n = n0 + j * 8;
+                    float b[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    float r[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    if (n < p.N) {
+                        if (p.bias != nullptr) {
+                            const uint4 bv = __ldg(reinterpret_cast<const uint4*>(p.bias + n));
+                            b[0] = bf16_lo_f(bv.x); b[1] = bf16_hi_f(bv.x);
+                            b[2] = bf16_lo_f(bv.y); b[3] = bf16_hi_f(bv.y);
+                            b[4] = bf16_lo_f(bv.z); b[5] = bf16_hi_f(bv.z);
+                            b[6] = bf16_lo_f(bv.w); b[7] = bf16_hi_f(bv.w);
+                        }
+                        if (p.residual != nullptr && row_ok) {
+                            const uint4 rv = __ldg(reinterpret_cast<const uint4*>(p.residual + row * p.ldr + n));
+                            r[0] = bf16_lo_f(rv.x); r[1] = bf16_hi_f(rv.x);
+                            r[2] = bf16_lo_f(rv.y); r[3] = bf16_hi_f(rv.y);
+                            r[4] = bf16_lo_f(rv.z); r[5] = bf16_hi_f(rv.z);
+                            r[6] = bf16_lo_f(rv.w); r[7] = bf16_hi_f(rv.w);
+                        }
+                    }
+                    uint32_t o[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float y0 = fmaf(s, __uint_as_float(v[j * 8 + 2 * e]), b[2 * e]) + r[2 * e];
+                        const float y1 = fmaf(s, __uint_as_float(v[j * 8 + 2 * e + 1]), b[2 * e + 1]) + r[2 * e + 1];
+                        o[e] = pack_bf16x2(y0, y1);
+                    }
+                    // 128-byte rows, 16-byte chunk index XOR (row % 8): the 128-byte swizzle
+                    sts128(cbuf + lane * 128 + ((j ^ (lane & 7)) << 4), o[0], o[1], o[2], o[3]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&tmap_y, n0, m0, cbuf);
+                    tma_store_commit();
+                }
+                cb = (cb + 1 == Cfg::CBUFS) ? 0 : cb + 1;
+            }
+        }
+        if (lane == 0) tma_store_wait_all<0>();
+    }
+
+    // ---------------------------------------------------------------------- teardown ----------
+    tc_fence_before();
+    __syncthreads();
+    if constexpr (CG == 2) cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc<CG>(tmem_base, Cfg::TMEM_COLS);
+    }
+}
+
+}  // namespace lynx
