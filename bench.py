@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the 2:4 activation-sparse linear layer (prune/compress + sparse GEMM + epilogue).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one pass of the whole hot path over one batch of synthetic activations:
+``lynx_prune_compress`` (Top-2-of-4 selection, compression, per-row norm-compensation scale)
+followed by ``lynx_sparse_linear`` (tcgen05 sparse GEMM with scale + bias epilogue), i.e. the two
+launches of the SEPARATE mode of ``lynx_act_sparse_linear``.  Prints ONE JSON line.
+
+* ``value``   dense-equivalent TFLOP/s (2*M*N*K per step) with inputs resident in HBM.
+* ``e2e``     same metric through ``lynx_act_sparse_linear_host`` (pinned host X in, host Y out).
+* ``roofline`` for the dominant kernel (the sparse GEMM), timed live with CUDA events inside the
+  timed region; ``roofline_prune`` for the HBM-bound prune/compress kernel.
+* ``cpu_baseline`` the CPU oracle, as it stands, on a bounded sample of rows of the same workload.
+* ``--impl reference`` times the CPU oracle only (there is no other reference implementation).
+
+Multi-GPU (``--gpus N`` under torchrun): the path does not shard; every rank runs an independent
+replica on its own GPU and the aggregate is reported ("replicas only", weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "2:4-act linear TFLOP/s (dense-equiv) and speedup vs dense bf16 GEMM, 1xB200"
+UNIT = "TFLOP/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse GEMM kernel on the
+# mlp_down workload, from the ncu capture summarised in profiles/ (None until captured).
+NCU_TRAFFIC_BYTES = {"mlp_down": None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mlp_down")
+    ap.add_argument("--comp", default="row", choices=["none", "row", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        try:
+            proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                     "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                    stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            return
+        try:
+            while not self._stop.is_set():
+                line = proc.stdout.readline()
+                if not line:
+                    break
+                self.samples.append((time.time(), [x.strip() for x in line.split(",")]))
+        finally:
+            proc.terminate()
+
+    def start(self):
+        self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        self._thread.join(timeout=3)
+
+    def summary(self, t0: float, t1: float):
+        rows = [s for (t, s) in self.samples if t0 <= t <= t1 + 0.15] or [s for (_, s) in self.samples]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": float(rows[0][1]),
+                "power_w_max": max(float(r[2]) for r in rows), "reasons": sorted(reasons), "samples": len(rows)}
+
+
+def max_over_ranks(ms: float, world: int, device: str = "cuda") -> float:
+    """Slowest rank's time: replicas run independently, the job is as slow as its slowest rank."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tflops(flops_per_step: float, steps: int, total_ms: float, world: int) -> float:
+    """Whole-job dense-equivalent TFLOP/s of `world` independent replicas."""
+    return flops_per_step * steps * world / (total_ms * 1e-3) / 1e12
+
+
+def oracle_sample_rate(wl, comp_mode, target_seconds=15.0):
+    """Times the CPU oracle on a bounded sample of rows of the workload.  -> dict for the JSON."""
+    import numpy as np
+
+    import oracle
+    from paper_2605_26632_b200 import inputs
+
+    cores = oracle.num_threads()
+    rows_small = max(8, cores)
+    # generate only as many rows of X as the largest sample can use; W in full
+    max_rows = min(wl.M, max(rows_small * 64, 1024))
+    d = inputs.make_workload(wl, with_bias=True, M=max_rows)
+    X, W, b = inputs.as_u16(d["X"]), inputs.as_u16(d["W"]), inputs.as_u16(d["bias"])
+    t0 = time.perf_counter()
+    oracle.act_sparse_linear(X[:rows_small], W, bias=b, comp_mode=comp_mode)
+    dt = time.perf_counter() - t0
+    n_rows = int(min(max_rows, max(rows_small, rows_small * target_seconds / max(dt, 1e-3))))
+    n_rows = max(rows_small, (n_rows // cores) * cores)
+    t0 = time.perf_counter()
+    oracle.act_sparse_linear(X[:n_rows], W, bias=b, comp_mode=comp_mode)
+    dt = time.perf_counter() - t0
+    tflops = 2.0 * n_rows * wl.N * wl.K / dt / 1e12
+    return {"value": tflops, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n_rows} of {wl.M} rows of {wl.name} (all N={wl.N} outputs, full K={wl.K}), "
+                      f"{dt:.1f} s wall", "seconds": dt, "rows": n_rows}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, as it stands, on bounded samples (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2605_26632_b200 import inputs
+
+    import oracle
+
+    wl = inputs.WORKLOADS[args.workload]
+    comp_mode = {"none": 0, "row": 1, "tensor": 2}[args.comp]
+    oracle.build()
+    budget = 120.0  # seconds for the whole run
+    per_step = max(0.5, budget / max(1, args.steps + args.warmup))
+    cal = oracle_sample_rate(wl, comp_mode, target_seconds=min(per_step, 10.0))
+    rows = cal["rows"]
+    import numpy as np
+
+    d = inputs.make_workload(wl, with_bias=True, M=rows)
+    X, W, b = inputs.as_u16(d["X"]), inputs.as_u16(d["W"]), inputs.as_u16(d["bias"])
+    for _ in range(min(args.warmup, 2)):
+        oracle.act_sparse_linear(X, W, bias=b, comp_mode=comp_mode)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.act_sparse_linear(X, W, bias=b, comp_mode=comp_mode)
+    dt = time.perf_counter() - t0
+    tflops = 2.0 * rows * wl.N * wl.K * args.steps / dt / 1e12
+    cpu = {"value": tflops, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": f"each step = first {rows} of {wl.M} rows of {wl.name} (all N, full K)"}
+    out = {"impl": "reference", "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+           "data": "synthetic", "config": {"workload": wl.name, "M": wl.M, "K": wl.K, "N": wl.N,
+                                           "comp": args.comp, "rows_per_step": rows},
+           "cpu_baseline": cpu,
+           "e2e": {"value": tflops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_26632_b200 import binding, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    wl = inputs.WORKLOADS[args.workload]
+    comp_mode = {"none": 0, "row": 1, "tensor": 2}[args.comp]
+    M, K, N = wl.M, wl.K, wl.N
+    peaks = load_peaks()
+    lx = binding.Lynx(local_rank)
+    lx.reserve(M, N, K)
+
+    d = inputs.make_workload(wl, with_bias=True)
+    # Device-resident inputs, rotated over NSETS distinct copies so that, together with W, values,
+    # metadata and Y (>= 246 MB per step for mlp_down), nothing a step reads is left in the 126 MB L2
+    # by the previous step.
+    NSETS = 3
+    Xs = [d["X"].cuda() if i == 0 else None for i in range(NSETS)]
+    for i in range(1, NSETS):
+        Xs[i] = torch.roll(Xs[0], shifts=i * 4, dims=0).contiguous()
+    Ws = [d["W"].cuda() for _ in range(NSETS)]
+    bias = d["bias"].cuda()
+    vals = [torch.empty((M, K // 2), dtype=torch.bfloat16, device="cuda") for _ in range(NSETS)]
+    metas = [torch.empty(binding.meta_bytes(M, K), dtype=torch.uint8, device="cuda") for _ in range(NSETS)]
+    scales = [torch.empty(M, dtype=torch.float32, device="cuda") for _ in range(NSETS)]
+    Ys = [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(NSETS)]
+    stream = torch.cuda.current_stream()
+
+    def step(i, ev=None):
+        j = i % NSETS
+        if ev is not None:
+            ev[0].record(stream)
+        lx.prune_compress(Xs[j], comp_mode, vals[j], metas[j], scales[j] if comp_mode else None)
+        if ev is not None:
+            ev[1].record(stream)
+        lx.sparse_linear(vals[j], metas[j], Ws[j], bias, scales[j] if comp_mode else None, None, Ys[j])
+        if ev is not None:
+            ev[2].record(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    if lx.last_error() != 0:
+        raise SystemExit("device-side timeout during warm-up")
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = lx.launch_count()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i, evs[i])
+    e1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    launches = lx.launch_count() - launches0
+    total_ms = e0.elapsed_time(e1)
+    total_ms = max_over_ranks(total_ms, world)
+    prune_ms = [ev[0].elapsed_time(ev[1]) for ev in evs]
+    gemm_ms = [ev[1].elapsed_time(ev[2]) for ev in evs]
+
+    # dense bf16 GEMM of the same shape on the same GPU (same rotation, same event timing)
+    dense_out = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    for i in range(3):
+        torch.nn.functional.linear(Xs[i % NSETS], Ws[i % NSETS], bias, out=None)
+    torch.cuda.synchronize()
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d0.record(stream)
+    for i in range(args.steps):
+        dense_out = torch.nn.functional.linear(Xs[i % NSETS], Ws[i % NSETS], bias)
+    d1.record(stream)
+    torch.cuda.synchronize()
+    dense_ms = d0.elapsed_time(d1) / args.steps
+    t_wall2 = time.time()
+
+    # end to end through the host-buffer entry point: pinned X in, pinned Y out, every step
+    e2e = None
+    if not args.no_e2e:
+        xh = [d["X"].pin_memory(), torch.roll(d["X"], 4, 0).contiguous().pin_memory()]
+        yh = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+        for i in range(2):
+            lx.act_sparse_linear_host(xh[i % 2], Ws[0], bias, comp_mode, yh)
+        e2e_steps = max(3, min(args.steps, 20))
+        barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for i in range(e2e_steps):
+            lx.act_sparse_linear_host(xh[i % 2], Ws[i % NSETS], bias, comp_mode, yh)
+        h1.record(stream)
+        barrier()
+        e2e_ms = h0.elapsed_time(h1)
+        e2e_ms = max_over_ranks(e2e_ms, world)
+        e2e = {"value": aggregate_tflops(2.0 * M * N * K, e2e_steps, e2e_ms, world), "unit": UNIT,
+               "h2d_bytes_per_step": M * K * 2, "d2h_bytes_per_step": M * N * 2, "steps": e2e_steps,
+               "ms_per_step": e2e_ms / e2e_steps}
+    sampler.stop()
+    if lx.last_error() != 0:
+        raise SystemExit("device-side timeout during the timed region")
+
+    flops = 2.0 * M * N * K
+    ms_per_step = total_ms / args.steps
+    value = aggregate_tflops(flops, args.steps, total_ms, world)
+    gemm_avg_ms = sum(gemm_ms) / len(gemm_ms)
+    prune_avg_ms = sum(prune_ms) / len(prune_ms)
+    sparse_peak = 2.0 * peaks["bf16_tflops_sustained"]
+    gemm_tf = flops / (gemm_avg_ms * 1e-3) / 1e12
+    prune_bytes = M * K * 3.125 + (4 * M if comp_mode else 0)
+    prune_gbs = prune_bytes / (prune_avg_ms * 1e-3) / 1e9
+    clocks = sampler.summary(t_wall0, t_wall1)
+    clocks_dense = sampler.summary(t_wall1, t_wall2)
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "M": M, "K": K, "N": N, "comp": args.comp, "fuse": "separate",
+                   "parallelism": "replicas only" if world > 1 else "single gpu",
+                   "l2": f"inputs larger than L2: {NSETS} rotating copies of X/W/values/metadata/Y, "
+                         f"{(M*K*2 + N*K*2 + M*K + M*K//8 + M*N*2)/1e6:.0f} MB touched per step"},
+        "speedup_vs_dense_bf16": dense_ms / ms_per_step,
+        "dense_bf16": {"ms": dense_ms, "tflops": flops / (dense_ms * 1e-3) / 1e12, "impl": "torch F.linear (cuBLASLt)",
+                       "sm_mhz": clocks_dense.get("sm_mhz")},
+        "kernels": {"prune_compress_ms": prune_avg_ms, "sparse_gemm_ms": gemm_avg_ms},
+        "roofline": {"bound": "tensor", "kernel": "sparse_gemm_kernel", "achieved": gemm_tf, "peak": sparse_peak,
+                     "unit": "TFLOP/s", "frac": gemm_tf / sparse_peak,
+                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
+                     "peak_kind": f"2 x bf16_tflops_sustained ({peaks['source']}); dense-equivalent flops",
+                     "frac_of_burst_peak": gemm_tf / (2.0 * peaks["bf16_tflops"])},
+        "roofline_prune": {"bound": "hbm", "kernel": "prune_compress_kernel", "achieved": prune_gbs,
+                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": prune_gbs / peaks["hbm_gbs"],
+                           "frac_of_8TBs_nominal": prune_gbs / 8000.0, "bytes_per_launch": prune_bytes,
+                           "peak_kind": f"hbm_gbs ({peaks['source']})"},
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+
+        oracle.build()
+        out["cpu_baseline"] = {k: v for k, v in oracle_sample_rate(wl, comp_mode).items() if k not in ("seconds", "rows")}
+    elif rank == 0:
+        out["cpu_baseline"] = None
+
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,303 @@
+"""GPU parity tests: the CUDA path (through the C ABI) against the CPU oracle.
+
+Bars: selection masks, values and metadata bit-exact; row scale within 1e-5 relative (fp32 sums in
+a different order than the oracle's fp64 sums); Y within relative Frobenius error 5e-3 and
+max |dY| <= 2e-2 * max |Y_ref| of the oracle's fp32 result.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_26632_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+RFE_TOL = 5e-3
+MAXABS_TOL = 2e-2
+SCALE_RTOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def lx():
+    from paper_2605_26632_b200 import binding
+
+    ctx = binding.Lynx(0)
+    yield ctx
+    torch.cuda.synchronize()
+    assert ctx.last_error() == 0
+    ctx.close()
+
+
+def u16(t):
+    return inputs.as_u16(t.detach().cpu())
+
+
+def check_y(Y, ref):
+    yf = Y.float().cpu().numpy()
+    rfe = np.linalg.norm(yf - ref) / max(np.linalg.norm(ref), 1e-30)
+    mx = np.abs(yf - ref).max() / max(np.abs(ref).max(), 1e-30)
+    assert rfe <= RFE_TOL, f"relative Frobenius error {rfe}"
+    assert mx <= MAXABS_TOL, f"max abs error ratio {mx}"
+    return rfe, mx
+
+
+def check_compressed(lx, X, values, meta, scale=None, mode=0):
+    """values / metadata (hardware order and canonical) / decompression, all bit-exact."""
+    M, K = X.shape
+    Xu = u16(X)
+    ov, om = oracle.compress(Xu)
+    assert (u16(values) == ov).all(), "values differ"
+    assert (meta.cpu().numpy() == oracle.meta_canon_to_hw(om, M, K)).all(), "hardware metadata differs"
+    canon = lx.meta_to_canonical(meta, M, K).cpu().numpy().view(np.uint16)
+    assert (canon == om).all(), "canonical metadata differs"
+    dec = u16(lx.decompress(values, meta))
+    assert (dec == Xu * oracle.topk24_mask(Xu)).all(), "decompress(compress(X)) != mask * X"
+    if mode:
+        np.testing.assert_allclose(scale.cpu().numpy(), oracle.row_scale(Xu, mode), rtol=SCALE_RTOL)
+    return ov, om
+
+
+# ------------------------------------------------------------------ prune / compress -----------
+
+@pytest.mark.parametrize("M,K,dist,mode", [
+    (256, 512, "gelu", 1),        # the tiny configuration
+    (1, 128, "normal", 1),        # single row, single K block
+    (17, 256, "outlier", 2),      # ragged 16-row block
+    (200, 384, "gelu_chan", 1),   # ragged 128-row block, K not a multiple of 1024
+    (300, 1024, "normal", 0),
+    (1000, 3072, "outlier", 2),
+])
+def test_prune_compress_matches_oracle(lx, M, K, dist, mode):
+    X = inputs.make_x(M, K, dist, 100 + M).cuda()
+    values, meta, scale = lx.prune_compress(X, mode)
+    check_compressed(lx, X, values, meta, scale, mode)
+
+
+def test_prune_compress_strided_input(lx):
+    M, K = 96, 256
+    big = inputs.make_x(M, 512, "normal", 5).cuda()
+    X = big[:, 128:128 + K]  # ldx = 512, 32-byte aligned start
+    values, meta, scale = lx.prune_compress(X, 1)
+    check_compressed(lx, X.contiguous(), values, meta, scale, 1)
+
+
+def test_prune_compress_special_values(lx):
+    """NaN, +-Inf, +-0 and subnormals rank by their 15 magnitude bits; ties go to the lower index."""
+    rng = np.random.default_rng(1)
+    pool = np.array([0x0000, 0x8000, 0x7FC0, 0xFFC1, 0x7F80, 0xFF80, 0x0001, 0x8001, 0x007F, 0x3F80, 0xBF80,
+                     0x3F81, 0x4000, 0x7F7F], dtype=np.uint16)
+    Xn = pool[rng.integers(0, len(pool), size=(64, 256))]
+    X = inputs.from_u16(Xn).cuda()
+    values, meta, _ = lx.prune_compress(X, 0)
+    ov, om = oracle.compress(Xn)
+    assert (u16(values) == ov).all()
+    assert (meta.cpu().numpy() == oracle.meta_canon_to_hw(om, 64, 256)).all()
+
+
+def test_prune_compress_all_bit_patterns(lx):
+    rng = np.random.default_rng(2)
+    Xn = rng.integers(0, 1 << 16, size=(128, 512), dtype=np.uint16)
+    X = inputs.from_u16(Xn).cuda()
+    values, meta, _ = lx.prune_compress(X, 0)
+    ov, om = oracle.compress(Xn)
+    assert (u16(values) == ov).all()
+    assert (meta.cpu().numpy() == oracle.meta_canon_to_hw(om, 128, 512)).all()
+
+
+def test_prune_compress_is_deterministic(lx):
+    X = inputs.make_x(512, 1024, "gelu", 9).cuda()
+    a = lx.prune_compress(X, 1)
+    b = lx.prune_compress(X, 1)
+    for s, t in zip(a, b):
+        assert torch.equal(s, t)
+
+
+# ------------------------------------------------------------------ silicon pins of the layout --
+
+@pytest.mark.parametrize("M,K", [(128, 128), (256, 512), (300, 1024)])
+def test_identity_weight_returns_masked_x_exactly(lx, M, K):
+    """W = I: every product is x*1 and every other addend is 0, so Y must equal mask*X bit for bit
+    (up to the sign of zero).  Any error in the metadata or value layout shows here."""
+    X = inputs.make_x(M, K, "normal", 3).cuda()
+    values, meta, _ = lx.prune_compress(X, 0)
+    W = torch.eye(K, dtype=torch.bfloat16, device="cuda")
+    Y = lx.sparse_linear(values, meta, W)
+    Xu = u16(X)
+    want = oracle.bf16_to_f32(Xu * oracle.topk24_mask(Xu))
+    assert (Y.float().cpu().numpy() == want).all()
+
+
+def test_one_hot_probes(lx):
+    M, K = 128, 256
+    W = torch.eye(K, dtype=torch.bfloat16, device="cuda")
+    for (m, k) in [(0, 0), (7, 3), (8, 17), (15, 31), (16, 32), (64, 127), (127, 255), (33, 130)]:
+        X = torch.zeros(M, K, dtype=torch.bfloat16)
+        X[m, k] = 2.0
+        values, meta, _ = lx.prune_compress(X.cuda(), 0)
+        Y = lx.sparse_linear(values, meta, W).float().cpu()
+        assert Y[m, k] == 2.0 and Y.abs().sum() == 2.0, (m, k)
+
+
+# ------------------------------------------------------------------ product + epilogue ---------
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("with_bias,with_res", [(False, False), (True, False), (True, True)])
+def test_tiny_config_full_oracle(lx, mode, with_bias, with_res):
+    wl = inputs.WORKLOADS["tiny"]
+    d = inputs.make_workload(wl, with_bias=with_bias, with_residual=with_res)
+    X, W = d["X"].cuda(), d["W"].cuda()
+    b = d["bias"].cuda() if with_bias else None
+    r = d["residual"].cuda() if with_res else None
+    ref = oracle.act_sparse_linear(u16(X), u16(W), bias=None if b is None else u16(b), comp_mode=mode,
+                                   Yr=None if r is None else u16(r))
+    # separate calls
+    values, meta, scale = lx.prune_compress(X, mode)
+    check_compressed(lx, X, values, meta, scale, mode)
+    Y = lx.sparse_linear(values, meta, W, b, scale, r)
+    check_y(Y, ref["Y"])
+    # one call
+    Y2 = lx.act_sparse_linear(X, W, b, mode, r)
+    check_y(Y2, ref["Y"])
+    assert torch.equal(Y, Y2)
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6])
+def test_every_tile_configuration(cfg, monkeypatch):
+    """All compiled tile shapes (one- and two-CTA MMAs, 128/192/256 columns) give the same answer."""
+    from paper_2605_26632_b200 import binding
+
+    monkeypatch.setenv("LYNX_GEMM_CFG", str(cfg))
+    ctx = binding.Lynx(0)
+    try:
+        wl = inputs.Workload("t", 300, 640, 456, "outlier", 77)  # ragged M, N not a tile multiple
+        d = inputs.make_workload(wl, with_bias=True, with_residual=True)
+        X, W, b, r = d["X"].cuda(), d["W"].cuda(), d["bias"].cuda(), d["residual"].cuda()
+        ref = oracle.act_sparse_linear(u16(X), u16(W), bias=u16(b), comp_mode=1, Yr=u16(r))
+        Y = ctx.act_sparse_linear(X, W, b, 1, r)
+        check_y(Y, ref["Y"])
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 128, 8), (5, 256, 72), (129, 384, 200), (257, 128, 1000)])
+def test_ragged_shapes(lx, M, K, N):
+    wl = inputs.Workload("t", M, K, N, "normal", 31)
+    d = inputs.make_workload(wl, with_bias=True, with_residual=True)
+    X, W, b, r = d["X"].cuda(), d["W"].cuda(), d["bias"].cuda(), d["residual"].cuda()
+    ref = oracle.act_sparse_linear(u16(X), u16(W), bias=u16(b), comp_mode=1, Yr=u16(r))
+    Y = lx.act_sparse_linear(X, W, b, 1, r)
+    check_y(Y, ref["Y"])
+
+
+def test_integer_valued_inputs_are_exact(lx):
+    """Small integers: every partial sum is exact in fp32 and in bf16, so Y must equal the oracle."""
+    rng = np.random.default_rng(4)
+    M, K, N = 256, 512, 256
+    X = torch.from_numpy(rng.integers(-4, 5, size=(M, K)).astype(np.float32)).to(torch.bfloat16)
+    W = torch.from_numpy(rng.integers(-1, 2, size=(N, K)).astype(np.float32)).to(torch.bfloat16)
+    ref = oracle.act_sparse_linear(u16(X), u16(W))
+    assert np.abs(ref["Y"]).max() <= 256  # exactly representable in bf16
+    Y = lx.act_sparse_linear(X.cuda(), W.cuda())
+    assert (Y.float().cpu().numpy() == ref["Y"]).all()
+
+
+def test_already_sparse_input_equals_dense_linear(lx):
+    """X already 2:4 sparse: the layer is an ordinary linear layer (library reference, fp32)."""
+    g = torch.Generator().manual_seed(8)
+    M, K, N = 384, 1024, 320
+    x = torch.randn(M, K, generator=g)
+    keep = torch.zeros(M, K // 4, 4, dtype=torch.bool)
+    pos = torch.rand(M, K // 4, 4, generator=g).argsort(-1)[..., :2]
+    keep.scatter_(-1, pos, True)
+    x = torch.where(keep.reshape(M, K), x + torch.sign(x), torch.zeros(())).to(torch.bfloat16)
+    w = inputs.make_w(N, K, 8)
+    b = inputs.make_bias(N, 8)
+    Y = lx.act_sparse_linear(x.cuda(), w.cuda(), b.cuda(), 1)
+    ref = torch.nn.functional.linear(x.float(), w.float(), b.float()).numpy()
+    check_y(Y, ref)
+
+
+def test_gemm_is_deterministic(lx):
+    wl = inputs.Workload("t", 1024, 1024, 768, "gelu", 12)
+    d = inputs.make_workload(wl)
+    X, W, b = d["X"].cuda(), d["W"].cuda(), d["bias"].cuda()
+    a = lx.act_sparse_linear(X, W, b, 1)
+    c = lx.act_sparse_linear(X, W, b, 1)
+    assert torch.equal(a, c)
+
+
+def test_host_buffer_entry_point(lx):
+    wl = inputs.WORKLOADS["tiny"]
+    d = inputs.make_workload(wl)
+    ref = oracle.act_sparse_linear(u16(d["X"]), u16(d["W"]), bias=u16(d["bias"]), comp_mode=1)
+    Y = lx.act_sparse_linear_host(d["X"].pin_memory(), d["W"].cuda(), d["bias"].cuda(), 1)
+    check_y(Y, ref["Y"])
+
+
+# ------------------------------------------------------------------ full-size workloads --------
+
+def _full_size_case(lx, wl, n_rows, mode=1):
+    d = inputs.make_workload(wl, with_bias=True)
+    X, W, b = d["X"].cuda(), d["W"].cuda(), d["bias"].cuda()
+    values, meta, scale = lx.prune_compress(X, mode)
+    Xu = u16(d["X"])
+    ov, om = oracle.compress(Xu)
+    assert (u16(values) == ov).all()
+    assert (meta.cpu().numpy() == oracle.meta_canon_to_hw(om, wl.M, wl.K)).all()
+    np.testing.assert_allclose(scale.cpu().numpy(), oracle.row_scale(Xu, mode), rtol=SCALE_RTOL)
+    Y = lx.sparse_linear(values, meta, W, b, scale)
+    rows = np.sort(np.random.default_rng(wl.seed).choice(wl.M, n_rows, replace=False)).astype(np.int64)
+    rows[0], rows[-1] = 0, wl.M - 1
+    ref = oracle.act_sparse_linear(Xu, u16(d["W"]), bias=u16(d["bias"]), comp_mode=mode, rows=rows)
+    check_y(Y[torch.from_numpy(rows).cuda()], ref["Y"])
+    # same launch configuration as the bench: the single-call path must agree bit for bit
+    Y2 = lx.act_sparse_linear(X, W, b, mode)
+    assert torch.equal(Y, Y2)
+
+
+@pytest.mark.parametrize("name", ["mlp_down", "attn_qkv", "attn_out", "mlp_up"])
+def test_dit_workloads_full_size(lx, name):
+    """Values and metadata checked on every element, Y on 48 sampled rows (all N columns)."""
+    _full_size_case(lx, inputs.WORKLOADS[name], 48)
+
+
+@pytest.mark.parametrize("M", inputs.SWEEP_M)
+@pytest.mark.parametrize("K,N", inputs.SWEEP_KN)
+def test_token_sweep(lx, M, K, N):
+    idx = inputs.SWEEP_M.index(M) * 4 + inputs.SWEEP_KN.index((K, N))
+    _full_size_case(lx, inputs.sweep_workload(M, K, N, idx), 16)
+
+
+# ------------------------------------------------------------------ host-side error reporting ---
+
+def test_argument_errors_are_reported_not_launched(lx):
+    from paper_2605_26632_b200 import binding
+
+    X = torch.zeros(16, 192, dtype=torch.bfloat16, device="cuda")  # K % 128 != 0
+    with pytest.raises(binding.LynxError) as e:
+        lx.prune_compress(X, 0, values=torch.empty(16, 96, dtype=torch.bfloat16, device="cuda"),
+                          meta=torch.empty(4096, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 2
+    X = torch.zeros(16, 256 + 8, dtype=torch.bfloat16, device="cuda")[:, 8:]  # misaligned rows
+    with pytest.raises(binding.LynxError) as e:
+        lx.prune_compress(X, 0)
+    assert e.value.status == 3
+    values = torch.zeros(16, 64, dtype=torch.bfloat16, device="cuda")
+    meta = torch.zeros(2048, dtype=torch.uint8, device="cuda")
+    W = torch.zeros(12, 128, dtype=torch.bfloat16, device="cuda")  # N % 8 != 0
+    with pytest.raises(binding.LynxError) as e:
+        lx.sparse_linear(values, meta, W)
+    assert e.value.status == 2
+    with pytest.raises(binding.LynxError) as e:  # scale requested but no buffer
+        lx._lib.lynx_prune_compress.restype = int
+        from ctypes import c_void_p
+        st = lx._lib.lynx_prune_compress(lx._h, c_void_p(values.data_ptr()), 16, 128, 128,
+                                         c_void_p(values.data_ptr()), c_void_p(meta.data_ptr()), None, 1, None)
+        binding._check(st, "prune")
+    assert e.value.status == 1
+    assert lx.last_error() == 0
