@@ -23,7 +23,8 @@ struct lynx_ctx {
     void* scratch = nullptr;  // compressed operands, scale, sums, host staging mirrors
     size_t scratch_bytes = 0;
     int64_t launches = 0;
-    int gemm_cfg = 0;  // 0 = auto
+    int gemm_cfg = 0;   // 0 = auto
+    int prune_tpu = 0;  // 0 = auto
     std::mutex mu;
 };
 
@@ -73,17 +74,23 @@ lynx_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? LYNX_OK : LYNX_ER
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Scratch layout for (M, N, K): [values][meta][row_scale M floats][sums 2M floats][X stage][Y stage]
+// Scratch layout for (M, N, K):
+// [partial row sums][sums 2M floats][values][meta][row_scale M floats][X stage][Y stage]
+// The first two sections serve lynx_prune_compress alone and come first so that a context that is
+// only used for pruning needs little memory.
 struct ScratchLayout {
-    size_t values, meta, scale, sums, xstage, ystage, total;
+    size_t partial, prune_end, values, meta, scale, sums, xstage, ystage, total;
 };
 ScratchLayout scratch_layout(int64_t M, int64_t N, int64_t K) {
     ScratchLayout L;
     size_t off = 0;
+    const size_t rb16 = (size_t)((M + 127) / 128) * 8, kblocks = (size_t)(K / 128);
+    L.partial = off; off = align_up(off + rb16 * kblocks * 32 * 4, 1024);
+    L.sums = off;    off = align_up(off + (size_t)M * 8, 1024);
+    L.prune_end = off;
     L.values = off; off = align_up(off + lynx_values_bytes(M, K), 1024);
     L.meta = off;   off = align_up(off + lynx_meta_bytes(M, K), 1024);
     L.scale = off;  off = align_up(off + (size_t)M * 4, 1024);
-    L.sums = off;   off = align_up(off + (size_t)M * 8, 1024);
     L.xstage = off; off = align_up(off + (size_t)M * K * 2, 1024);
     L.ystage = off; off = align_up(off + (size_t)M * N * 2, 1024);
     L.total = off;
@@ -150,7 +157,12 @@ lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int
                         int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp, void* Y, int64_t ldy,
                         cudaStream_t st) {
     int cfg = ctx->gemm_cfg;
-    if (cfg == 0) cfg = 1;
+    if (cfg == 0) {
+        // CTA-pair tiles.  Long K amortises the epilogue, so the single-accumulator 256 x 256 tile
+        // (fewest operand bytes per flop) wins; short K needs the epilogue hidden behind the next
+        // tile's main loop, which the double-buffered 256 x 192 tile provides.
+        cfg = (K >= 6144) ? 5 : 4;
+    }
 #define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, Y, ldy, st
     switch (cfg) {
         case 1: return launch_gemm_cfg<GemmCfg<128, 1, 4, 1>>(LYNX_GEMM_ARGS);
@@ -211,6 +223,8 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
     *ctx->err_host = DEV_OK;
     const char* env = getenv("LYNX_GEMM_CFG");  // development override of the tile configuration
     if (env) ctx->gemm_cfg = atoi(env);
+    env = getenv("LYNX_PRUNE_TPU");  // development override: 128-element K blocks per warp
+    if (env) ctx->prune_tpu = atoi(env);
     *out = ctx;
     return LYNX_OK;
 }
@@ -270,25 +284,44 @@ lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t
         return LYNX_ERR_ALIGNMENT;  // 32-byte vector accesses
     if ((s = check_device_error(ctx)) != LYNX_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // work decomposition: one warp per (16-row block, run of `tpu` K blocks)
+    const int64_t kblocks = K / 128;
+    const int64_t rb16 = ((M + 127) / 128) * 8;
+    int tpu = ctx->prune_tpu;
+    if (tpu <= 0) {
+        const int64_t resident = (int64_t)ctx->num_sms * 40;  // warps the GPU holds at ~48 registers
+        const int64_t want = (rb16 * kblocks) / (3 * resident);
+        tpu = (int)(want < 1 ? 1 : (want > 8 ? 8 : want));
+    }
+    while (kblocks % tpu) --tpu;
+    const int KS = (int)(kblocks / tpu);
     float* sums = nullptr;
-    if (mode == LYNX_COMP_TENSOR) {
+    float* partial = nullptr;
+    if (mode != LYNX_COMP_NONE) {
         std::lock_guard<std::mutex> lock(ctx->mu);
         ScratchLayout L = scratch_layout(M, 8, K);
-        if (ctx->scratch_bytes < L.sums + (size_t)M * 8) {
+        if (ctx->scratch_bytes < L.prune_end) {
             if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
         }
-        sums = reinterpret_cast<float*>(static_cast<char*>(ctx->scratch) + L.sums);
+        char* base = static_cast<char*>(ctx->scratch);
+        partial = reinterpret_cast<float*>(base + L.partial);
+        sums = reinterpret_cast<float*>(base + L.sums);
     }
-    const unsigned grid = (unsigned)(((M + 127) / 128) * (128 / PRUNE_ROWS));
+    const int64_t units = rb16 * KS;
+    const unsigned grid = (unsigned)((units + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS);
     if (mode == LYNX_COMP_NONE)
-        prune_compress_kernel<false><<<grid, PRUNE_THREADS, 0, st>>>(
+        prune_compress_kernel<false><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
             static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
-            row_scale, nullptr, 0);
+            row_scale, nullptr, nullptr, 0, tpu, KS, units);
     else
-        prune_compress_kernel<true><<<grid, PRUNE_THREADS, 0, st>>>(
+        prune_compress_kernel<true><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
             static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
-            row_scale, sums, (int)mode);
+            row_scale, sums, partial, (int)mode, tpu, KS, units);
     ctx->launches++;
+    if (mode != LYNX_COMP_NONE && KS > 1) {
+        row_scale_kernel<<<(unsigned)((M + 15) / 16), 256, 0, st>>>(partial, M, KS, (int)mode, row_scale, sums);
+        ctx->launches++;
+    }
     if (mode == LYNX_COMP_TENSOR) {
         tensor_scale_kernel<<<1, 1024, 0, st>>>(sums, M, row_scale);
         ctx->launches++;

@@ -2,8 +2,8 @@
 // compression to (values, 2-bit index metadata in sparse-MMA order) and the per-row sums the
 // norm-compensation scale needs -- one streaming pass over X.
 //
-// Work split: one CTA owns 16 rows (the row span of one 256-byte metadata slab); its warps take
-// 128-element K blocks round-robin.  Inside a block a lane owns 32 consecutive elements of row
+// Work split: one warp owns 16 rows (the row span of one 256-byte metadata slab) and a run of
+// 128-element K blocks.  Inside a block a lane owns 32 consecutive elements of row
 // r = lane/4 and of row r + 8, i.e. exactly the elements whose metadata make up the two 32-bit
 // words this lane writes, so no metadata bit ever crosses lanes:
 //     word(half h, lane) at slab byte h*128 + lane*4 = [row r : 16 bits][row r+8 : 16 bits]
@@ -19,8 +19,6 @@
 namespace lynx {
 
 constexpr int PRUNE_ROWS = 16;
-constexpr int PRUNE_WARPS = 8;
-constexpr int PRUNE_THREADS = PRUNE_WARPS * 32;
 
 // bitwise majority of three words
 __device__ __forceinline__ uint32_t maj3(uint32_t a, uint32_t b, uint32_t c) {
@@ -63,10 +61,28 @@ __device__ __forceinline__ uint32_t prune_lut_entry(uint32_t pattern, int j) {
     return sel | ((i0 | (i1 << 2)) << (16 + 4 * j));
 }
 
+// acc + lo^2 + hi^2 for the two bf16 halves of r: mixed-precision FMAs (bf16 x bf16 + fp32), the
+// products are exact in fp32 and every add rounds once.
+__device__ __forceinline__ float fma_sq_bf16x2(uint32_t r, float acc) {
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\t"
+        "fma.rn.f32.bf16 %0, lo, lo, %0;\n\tfma.rn.f32.bf16 %0, hi, hi, %0;\n\t}"
+        : "+f"(acc)
+        : "r"(r));
+    return acc;
+}
+
+__device__ __forceinline__ void write_scale_or_sums(int mode, int64_t m, float num, float den,
+                                                    float* row_scale, float* sums) {
+    if (mode == 1) row_scale[m] = sqrtf(num / (den + 1e-8f));
+    else {
+        sums[2 * m] = num;
+        sums[2 * m + 1] = den;
+    }
+}
+
 // One 32-byte vector = 16 consecutive elements = 4 groups -> 4 value registers + 16 metadata bits.
-template <bool SUMS>
 __device__ __forceinline__ uint32_t prune_vec16(const uint32_t (&r)[8], const uint32_t* lut,
-                                                uint32_t* v /*[4]*/, float& num, float& den) {
+                                                uint32_t* v /*[4]*/) {
     const uint32_t p01 = keep_patterns_x2(r[0], r[1], r[2], r[3]);
     const uint32_t p23 = keep_patterns_x2(r[4], r[5], r[6], r[7]);
     const char* base = reinterpret_cast<const char*>(lut);
@@ -78,75 +94,119 @@ __device__ __forceinline__ uint32_t prune_vec16(const uint32_t (&r)[8], const ui
     v[1] = prmt(r[2], r[3], e1);
     v[2] = prmt(r[4], r[5], e2);
     v[3] = prmt(r[6], r[7], e3);
-    if constexpr (SUMS) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float lo = bf16_lo_f(r[i]), hi = bf16_hi_f(r[i]);
-            num = fmaf(lo, lo, num);
-            num = fmaf(hi, hi, num);
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float lo = bf16_lo_f(v[i]), hi = bf16_hi_f(v[i]);
-            den = fmaf(lo, lo, den);
-            den = fmaf(hi, hi, den);
-        }
-    }
     return (e0 | e1 | e2 | e3) >> 16;
 }
 
-// mode: 0 none (row_scale written as 1 if non-null), 1 per-row scale, 2 partial sums for the
+// Work unit of one warp: 16 rows x (tiles_per_unit * 128) elements; the KS = kblocks /
+// tiles_per_unit units of a 16-row block are independent warps (many small CTAs keep the SMs'
+// load queues full).  With KS > 1 each unit writes its partial row sums
+// (partial[(rb16*KS + ks)*32 + 2*row + {0: sum x^2, 1: sum kept x^2}]) and row_scale_kernel adds
+// them in fixed order, so the result does not depend on scheduling.
+//
+// mode: 0 none (row_scale written as 1 if non-null), 1 per-row scale, 2 per-row sums for the
 // whole-tensor scale (sums[2*m] = sum x^2, sums[2*m+1] = sum kept x^2).
+#ifndef LYNX_PRUNE_CTA_WARPS
+#define LYNX_PRUNE_CTA_WARPS 4
+#endif
+#ifndef LYNX_PRUNE_MIN_CTAS
+#define LYNX_PRUNE_MIN_CTAS 1
+#endif
+constexpr int PRUNE_CTA_WARPS = LYNX_PRUNE_CTA_WARPS;
+
+template <bool SUMS, bool GUARD>
+__device__ __forceinline__ void prune_tile(const uint16_t* xa, const uint16_t* xb, uint16_t* va, uint16_t* vb,
+                                           uint32_t* slab, bool okA, bool okB, const uint32_t* lut, float& numA,
+                                           float& denA, float& numB, float& denB) {
+    uint32_t a0[8], a1[8], b0[8], b1[8];
+    if constexpr (GUARD) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a0[i] = a1[i] = b0[i] = b1[i] = 0u;
+        if (okA) {
+            ldg256_stream(xa, a0);
+            ldg256_stream(xa + 16, a1);
+        }
+        if (okB) {
+            ldg256_stream(xb, b0);
+            ldg256_stream(xb + 16, b1);
+        }
+    } else {
+        ldg256_stream(xa, a0);
+        ldg256_stream(xa + 16, a1);
+        ldg256_stream(xb, b0);
+        ldg256_stream(xb + 16, b1);
+    }
+    uint32_t oa[8], ob[8];
+    const uint32_t ma0 = prune_vec16(a0, lut, oa);
+    const uint32_t ma1 = prune_vec16(a1, lut, oa + 4);
+    const uint32_t mb0 = prune_vec16(b0, lut, ob);
+    const uint32_t mb1 = prune_vec16(b1, lut, ob + 4);
+    if (!GUARD || okA) stg256(va, oa);
+    if (!GUARD || okB) stg256(vb, ob);
+    // rows past M prune to the pattern (0,1) = nibble 0x4, the documented padding
+    slab[0] = ma0 | (mb0 << 16);
+    slab[32] = ma1 | (mb1 << 16);
+    if constexpr (SUMS) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            numA = fma_sq_bf16x2(a0[i], numA);
+            numB = fma_sq_bf16x2(b0[i], numB);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            numA = fma_sq_bf16x2(a1[i], numA);
+            numB = fma_sq_bf16x2(b1[i], numB);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            denA = fma_sq_bf16x2(oa[i], denA);
+            denB = fma_sq_bf16x2(ob[i], denB);
+        }
+    }
+}
+
 template <bool SUMS>
-__global__ void __launch_bounds__(PRUNE_THREADS)
+__global__ void __launch_bounds__(PRUNE_CTA_WARPS * 32, LYNX_PRUNE_MIN_CTAS)
 prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int64_t ldx,
                       uint16_t* __restrict__ values, uint8_t* __restrict__ meta,
-                      float* __restrict__ row_scale, float* __restrict__ sums, int mode) {
+                      float* __restrict__ row_scale, float* __restrict__ sums,
+                      float* __restrict__ partial, int mode, int tiles_per_unit, int KS,
+                      int64_t num_units) {
     __shared__ uint32_t lut[4 * 16];
-    __shared__ float red[PRUNE_WARPS][PRUNE_ROWS][2];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid < 64) lut[tid] = prune_lut_entry(tid & 15, tid >> 4);
     __syncthreads();
 
-    const int64_t row0 = (int64_t)blockIdx.x * PRUNE_ROWS;
+    const int64_t unit = (int64_t)blockIdx.x * PRUNE_CTA_WARPS + warp;
+    if (unit >= num_units) return;
+    const int64_t rb16 = unit / KS;
+    const int ks = (int)(unit - rb16 * KS);
+    const int64_t row0 = rb16 * PRUNE_ROWS;
     const int r = lane >> 2, q = lane & 3;
     const int64_t rowA = row0 + r, rowB = rowA + 8;
-    const bool okA = rowA < M, okB = rowB < M;
     const int64_t kblocks = K / 128;
-    // metadata slab of this CTA inside block (row0/128, kb)
-    uint8_t* slab0 = meta + ((row0 / 128) * kblocks) * 2048 + ((row0 % 128) / 16) * 256 + lane * 4;
-    const uint16_t* xa = X + rowA * ldx + q * 32;
-    const uint16_t* xb = X + rowB * ldx + q * 32;
-    uint16_t* va = values + rowA * (K / 2) + q * 16;
-    uint16_t* vb = values + rowB * (K / 2) + q * 16;
+    const int64_t kb0 = (int64_t)ks * tiles_per_unit;
+    // metadata slab of this row block inside block (row0/128, kb)
+    uint32_t* slab = reinterpret_cast<uint32_t*>(meta + ((row0 / 128) * kblocks + kb0) * 2048 +
+                                                 ((row0 % 128) / 16) * 256 + lane * 4);
+    const uint16_t* xa = X + rowA * ldx + kb0 * 128 + q * 32;
+    const uint16_t* xb = xa + 8 * ldx;
+    uint16_t* va = values + rowA * (K / 2) + kb0 * 64 + q * 16;
+    uint16_t* vb = va + 8 * (K / 2);
 
     float numA = 0.f, denA = 0.f, numB = 0.f, denB = 0.f;
-    for (int64_t kb = warp; kb < kblocks; kb += PRUNE_WARPS) {
-        uint32_t a0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, a1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        uint32_t b0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, b1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        if (okA) {
-            ldg256_stream(xa + kb * 128, a0);
-            ldg256_stream(xa + kb * 128 + 16, a1);
-        }
-        if (okB) {
-            ldg256_stream(xb + kb * 128, b0);
-            ldg256_stream(xb + kb * 128 + 16, b1);
-        }
-        uint32_t oa[8], ob[8];
-        const uint32_t ma0 = prune_vec16<SUMS>(a0, lut, oa, numA, denA);
-        const uint32_t ma1 = prune_vec16<SUMS>(a1, lut, oa + 4, numA, denA);
-        const uint32_t mb0 = prune_vec16<SUMS>(b0, lut, ob, numB, denB);
-        const uint32_t mb1 = prune_vec16<SUMS>(b1, lut, ob + 4, numB, denB);
-        if (okA) stg256(va + kb * 64, oa);
-        if (okB) stg256(vb + kb * 64, ob);
-        // rows past M prune to the pattern (0,1) = nibble 0x4, the documented padding
-        uint32_t* slab = reinterpret_cast<uint32_t*>(slab0 + kb * 2048);
-        slab[0] = ma0 | (mb0 << 16);
-        slab[32] = ma1 | (mb1 << 16);
+    if (row0 + PRUNE_ROWS <= M) {
+        for (int t = 0; t < tiles_per_unit; ++t)
+            prune_tile<SUMS, false>(xa + t * 128, xb + t * 128, va + t * 64, vb + t * 64, slab + t * 512, true,
+                                    true, lut, numA, denA, numB, denB);
+    } else {
+        const bool okA = rowA < M, okB = rowB < M;
+        for (int t = 0; t < tiles_per_unit; ++t)
+            prune_tile<SUMS, true>(xa + t * 128, xb + t * 128, va + t * 64, vb + t * 64, slab + t * 512, okA,
+                                   okB, lut, numA, denA, numB, denB);
     }
 
     if constexpr (SUMS) {
-        // the 4 lanes of a row, then the warps (fixed order: results are reproducible)
+        // the 4 lanes of a row
 #pragma unroll
         for (int off = 1; off <= 2; off <<= 1) {
             numA += __shfl_xor_sync(0xffffffffu, numA, off);
@@ -155,27 +215,49 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
             denB += __shfl_xor_sync(0xffffffffu, denB, off);
         }
         if (q == 0) {
-            red[warp][r][0] = numA;
-            red[warp][r][1] = denA;
-            red[warp][r + 8][0] = numB;
-            red[warp][r + 8][1] = denB;
-        }
-        __syncthreads();
-        if (tid < PRUNE_ROWS && row0 + tid < M) {
-            float num = 0.f, den = 0.f;
-#pragma unroll
-            for (int w = 0; w < PRUNE_WARPS; ++w) {
-                num += red[w][tid][0];
-                den += red[w][tid][1];
-            }
-            if (mode == 1) row_scale[row0 + tid] = sqrtf(num / (den + 1e-8f));
-            else {
-                sums[2 * (row0 + tid)] = num;
-                sums[2 * (row0 + tid) + 1] = den;
+            if (KS == 1) {
+                if (rowA < M) write_scale_or_sums(mode, rowA, numA, denA, row_scale, sums);
+                if (rowB < M) write_scale_or_sums(mode, rowB, numB, denB, row_scale, sums);
+            } else {
+                float* mine = partial + (rb16 * KS + ks) * 32;
+                *reinterpret_cast<float2*>(mine + 2 * r) = make_float2(numA, denA);
+                *reinterpret_cast<float2*>(mine + 2 * (r + 8)) = make_float2(numB, denB);
             }
         }
     } else {
-        if (row_scale != nullptr && tid < PRUNE_ROWS && row0 + tid < M) row_scale[row0 + tid] = 1.0f;
+        if (row_scale != nullptr && ks == 0 && lane < 16 && row0 + lane < M) row_scale[row0 + lane] = 1.0f;
+    }
+}
+
+// One CTA per 16-row block: adds the KS partial sums of each row in a fixed order (16 strided
+// running sums per row, then those 16 in ascending order), so the result is reproducible.
+__global__ void __launch_bounds__(256)
+row_scale_kernel(const float* __restrict__ partial, int64_t M, int KS, int mode, float* __restrict__ row_scale,
+                 float* __restrict__ sums) {
+    __shared__ float2 red[16][16];
+    const int row = threadIdx.x & 15, jl = threadIdx.x >> 4;
+    const int64_t rb16 = blockIdx.x;
+    const float2* p = reinterpret_cast<const float2*>(partial) + rb16 * KS * 16 + row;
+    float num = 0.f, den = 0.f;
+    for (int j = jl; j < KS; j += 16) {
+        const float2 v = __ldcg(p + j * 16);
+        num += v.x;
+        den += v.y;
+    }
+    red[jl][row] = make_float2(num, den);
+    __syncthreads();
+    if (threadIdx.x < 16) {
+        const int64_t m = rb16 * 16 + threadIdx.x;
+        if (m < M) {
+            num = 0.f;
+            den = 0.f;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                num += red[j][threadIdx.x].x;
+                den += red[j][threadIdx.x].y;
+            }
+            write_scale_or_sums(mode, m, num, den, row_scale, sums);
+        }
     }
 }
 

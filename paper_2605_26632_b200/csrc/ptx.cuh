@@ -275,7 +275,7 @@ __device__ __forceinline__ uint64_t make_desc_rows16(uint32_t smem_addr) {
 // ---------------------------------------------------------------------------- memory ---------
 
 __device__ __forceinline__ void ldg256_stream(const void* p, uint32_t (&r)[8]) {
-    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
                    "=r"(r[7])
                  : "l"(p));
