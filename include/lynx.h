@@ -119,6 +119,30 @@ LYNX_API lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M
                                          int64_t ldx, void* values, void* meta, float* row_scale,
                                          lynx_comp_mode mode, void* stream);
 
+/* Same operation as lynx_prune_compress for callers that cannot allocate device memory -- a
+ * serving process that has handed the whole device to its own memory pool (so cudaMalloc may
+ * fail or stall), or a latency-critical loop that must not hit the device-wide synchronisation
+ * cudaMalloc / cudaFree imply.  (The paper has no counterpart; this is a packaging variant.)
+ * It needs no context and calls no cudaMalloc, cudaFree or other allocating routine: the partial
+ * row sums and per-row sums that lynx_prune_compress keeps in its context's scratch live here in
+ * a fixed device array of LYNX_STATIC_SCRATCH_BYTES that is part of the library image (every GPU
+ * that loads the library holds it until the process exits).
+ *   - Works on the CURRENT device.  The first call on each device looks up the array's device
+ *     address (cudaGetSymbolAddress) and caches it; make that first call before any stream
+ *     capture begins.
+ *   - Shapes whose scratch need -- ceil(M/128)*8 * (K/128)/t * 128 bytes of partial sums, t the
+ *     K blocks per warp the library picks, plus 8*M bytes in LYNX_COMP_TENSOR mode -- exceeds
+ *     LYNX_STATIC_SCRATCH_BYTES are refused with LYNX_ERR_WORKSPACE; LYNX_COMP_NONE needs none.
+ *   - Every call shares the one array and finds the previous call's contents in it; nothing in
+ *     it has to start at zero (each call overwrites what it later reads).  Two calls that overlap
+ *     on the GPU (different streams, no ordering between them) race on it: order them.
+ *   - No device-side error word: the kernels involved have no waits that can time out.
+ * Arguments, layouts, alignment rules and results are exactly those of lynx_prune_compress. */
+#define LYNX_STATIC_SCRATCH_BYTES (8u << 20)
+LYNX_API lynx_status lynx_prune_compress_static(const void* X, int64_t M, int64_t K, int64_t ldx,
+                                                void* values, void* meta, float* row_scale,
+                                                lynx_comp_mode mode, void* stream);
+
 /* ---- step 5-6: 2:4 sparse x dense product and epilogue ---------------------------------------
  * (Algorithm 1 lines 5-6; Algorithm 2 for the bias.)
  *   Y[m, n] = bf16_rne( s_m * sum_k X~[m,k] W[n,k]  +  bias[n]  +  Y_r[m,n] )

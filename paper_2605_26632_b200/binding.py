@@ -21,7 +21,7 @@ EXPORTS = [
     "lynx_create", "lynx_destroy", "lynx_status_string", "lynx_last_error", "lynx_values_bytes",
     "lynx_meta_bytes", "lynx_workspace_bytes", "lynx_reserve", "lynx_prune_compress",
     "lynx_sparse_linear", "lynx_act_sparse_linear", "lynx_act_sparse_linear_host",
-    "lynx_meta_to_canonical", "lynx_decompress", "lynx_launch_count",
+    "lynx_meta_to_canonical", "lynx_decompress", "lynx_launch_count", "lynx_prune_compress_static",
 ]
 
 
@@ -71,6 +71,7 @@ def load_library() -> ctypes.CDLL:
     lib.lynx_act_sparse_linear_host.argtypes = [vp, vp, i64, i64, vp, i64, i64, vp, i32, vp, i32, vp]
     lib.lynx_meta_to_canonical.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.lynx_decompress.argtypes = [vp, vp, vp, i64, i64, vp, vp]
+    lib.lynx_prune_compress_static.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
     lib.lynx_launch_count.argtypes = [vp]
     lib.lynx_launch_count.restype = i64
     _lib = lib
@@ -106,6 +107,31 @@ def _bf16_2d(t: torch.Tensor, name: str):
     if t.dtype != torch.bfloat16 or t.dim() != 2 or t.stride(1) != 1:
         raise TypeError(f"{name}: expected a 2-D bf16 tensor with unit inner stride")
     return t
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def prune_compress_static(X: torch.Tensor, mode: int = COMP_NONE, values=None, meta=None, row_scale=None):
+    """``lynx_prune_compress_static``: the prune/compress step for callers that cannot allocate
+    device memory (a process whose memory pool owns the whole GPU, or a loop that must not incur
+    the device synchronisation an allocation implies).  The library allocates nothing: pass
+    ``values`` / ``meta`` / ``row_scale`` that you already own (they are only created here, with
+    torch, when left out).  Runs on the current device and torch's current stream, uses the
+    library's fixed scratch array shared by all calls -- do not overlap two calls on the GPU.
+    The first call on a device performs a one-time address look-up."""
+    _bf16_2d(X, "X")
+    M, K = X.shape
+    if values is None:
+        values = torch.empty((M, K // 2), dtype=torch.bfloat16, device=X.device)
+    if meta is None:
+        meta = torch.empty(meta_bytes(M, K), dtype=torch.uint8, device=X.device)
+    if row_scale is None and mode != COMP_NONE:
+        row_scale = torch.empty(M, dtype=torch.float32, device=X.device)
+    _check(load_library().lynx_prune_compress_static(_ptr(X), M, K, X.stride(0), _ptr(values), _ptr(meta),
+                                                     _ptr(row_scale), mode, _stream()),
+           "lynx_prune_compress_static")
+    return values, meta, row_scale
 
 
 class Lynx:

@@ -425,3 +425,84 @@ lynx_status lynx_decompress(lynx_ctx* ctx, const void* values, const void* meta,
 }
 
 }  // extern "C"
+
+// ================================================= entry point that allocates nothing ===========
+// Scratch for lynx_prune_compress_static: part of the library image, LYNX_STATIC_SCRATCH_BYTES
+// per GPU.  In host code this name is only a handle; the device address comes from
+// cudaGetSymbolAddress, looked up once per device (with that device current) and cached.
+static __device__ __align__(256) unsigned char g_static_scratch[LYNX_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int MAX_DEVICES = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[MAX_DEVICES] = {};
+int g_static_sms[MAX_DEVICES] = {};
+
+// device address of g_static_scratch on the current device (set-up on first use per device)
+lynx_status static_scratch_for_current_device(void** ptr, int* num_sms) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return LYNX_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return LYNX_ERR_CUDA;
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return LYNX_ERR_CUDA;
+        if (major != 10) return LYNX_ERR_UNSUPPORTED_ARCH;
+        g_static_sms[dev] = sms;
+        g_static_ptr[dev] = p;
+    }
+    *ptr = g_static_ptr[dev];
+    *num_sms = g_static_sms[dev];
+    return LYNX_OK;
+}
+}  // namespace
+
+extern "C" lynx_status lynx_prune_compress_static(const void* X, int64_t M, int64_t K, int64_t ldx, void* values,
+                                                  void* meta, float* row_scale, lynx_comp_mode mode, void* stream) {
+    if (M < 1 || K < 128) return LYNX_ERR_INVALID_ARG;
+    if (K % 128 != 0 || M > (1ll << 30) || K > (1ll << 30)) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    if (!X || !values || !meta) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW && mode != LYNX_COMP_TENSOR) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_NONE && !row_scale) return LYNX_ERR_INVALID_ARG;
+    if (ldx < K) return LYNX_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(X) & 31u) || (reinterpret_cast<uintptr_t>(values) & 31u) || !aligned16(meta) ||
+        (ldx % 16) != 0)
+        return LYNX_ERR_ALIGNMENT;
+    void* scratch = nullptr;
+    int num_sms = 0;
+    lynx_status s = static_scratch_for_current_device(&scratch, &num_sms);
+    if (s != LYNX_OK) return s;
+    // same work decomposition as lynx_prune_compress
+    const int64_t kblocks = K / 128;
+    const int64_t rb16 = ((M + 127) / 128) * 8;
+    const int64_t resident = (int64_t)num_sms * 40;
+    const int64_t want = (rb16 * kblocks) / (3 * resident);
+    int tpu = (int)(want < 1 ? 1 : (want > 8 ? 8 : want));
+    while (kblocks % tpu) --tpu;
+    const int KS = (int)(kblocks / tpu);
+    // static scratch: [partial sums: rb16 * KS * 32 floats][per-row sums: 2 * M floats]
+    const size_t partial_bytes = (mode != LYNX_COMP_NONE && KS > 1) ? (size_t)rb16 * KS * 32 * 4 : 0;
+    const size_t partial_padded = (partial_bytes + 255) / 256 * 256;
+    const size_t sums_bytes = (mode == LYNX_COMP_TENSOR) ? (size_t)M * 8 : 0;
+    if (partial_padded + sums_bytes > (size_t)LYNX_STATIC_SCRATCH_BYTES) return LYNX_ERR_WORKSPACE;
+    float* partial = reinterpret_cast<float*>(scratch);
+    float* sums = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + partial_padded);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t units = rb16 * KS;
+    const unsigned grid = (unsigned)((units + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS);
+    if (mode == LYNX_COMP_NONE)
+        prune_compress_kernel<false><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
+            static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
+            row_scale, nullptr, nullptr, 0, tpu, KS, units);
+    else
+        prune_compress_kernel<true><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
+            static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
+            row_scale, sums, partial, (int)mode, tpu, KS, units);
+    if (mode != LYNX_COMP_NONE && KS > 1)
+        row_scale_kernel<<<(unsigned)((M + 15) / 16), 256, 0, st>>>(partial, M, KS, (int)mode, row_scale, sums);
+    if (mode == LYNX_COMP_TENSOR) tensor_scale_kernel<<<1, 1024, 0, st>>>(sums, M, row_scale);
+    return cuda_ok(cudaGetLastError());
+}
