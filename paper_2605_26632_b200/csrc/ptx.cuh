@@ -208,6 +208,27 @@ __device__ __forceinline__ void mma_sp_bf16(uint32_t d_tmem, uint64_t a_desc, ui
             : "memory");
 }
 
+// Lean form for the issue loop: descriptors as (low word, shared high word), so that stepping
+// through a tile is one 32-bit add per operand.
+template <int CG>
+__device__ __forceinline__ void mma_sp_bf16_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                               uint32_t e_tmem, uint32_t idesc, uint32_t accumulate) {
+    if constexpr (CG == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], da, db, [%4], %5, p;\n\t}" ::"r"(d_tmem),
+            "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(e_tmem), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], da, db, [%4], %5, p;\n\t}" ::"r"(d_tmem),
+            "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(e_tmem), "r"(idesc), "r"(accumulate)
+            : "memory");
+}
+
 // 128 lanes x 128 bits, shared memory -> tensor memory (4 columns).
 template <int CG>
 __device__ __forceinline__ void tmem_cp_128x128b(uint32_t taddr, uint64_t s_desc) {

@@ -170,7 +170,13 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer --------
         if (leader && lane == 0) {
-            constexpr uint32_t idesc = make_idesc_sp_bf16(Cfg::BM * CG, BN);
+            constexpr uint32_t idesc0 = make_idesc_sp_bf16(Cfg::BM * CG, BN), idesc1 = idesc0 | 1u;
+            // descriptor words: low = start address (16-byte units) | LBO, high = SBO | version | swizzle
+            const uint64_t d0 = make_desc_sw128(sA);
+            const uint32_t desc_hi = (uint32_t)(d0 >> 32);
+            const uint32_t a_lo0 = (uint32_t)d0, b_lo0 = (uint32_t)make_desc_sw128(sB);
+            const uint64_t e_d0 = make_desc_rows16(sE);
+            constexpr uint32_t BH = Cfg::B_HALF_BYTES >> 4;
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             int it = 0;
@@ -180,6 +186,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, cta_abort, p.dev_error)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
+                uint32_t accumulate = 0;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, cta_abort, p.dev_error)) {
                         ok = false;
@@ -187,18 +194,16 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     }
                     tc_fence_after();
                     const uint32_t e_tmem = tmem_base + Cfg::E_COL0 + 4 * stage;
-                    tmem_cp_128x128b<CG>(e_tmem, make_desc_rows16(sE + stage * Cfg::E_BYTES));
-                    const uint64_t a_desc = make_desc_sw128(sA + stage * Cfg::A_BYTES);
-                    const uint64_t b_desc = make_desc_sw128(sB + stage * Cfg::B_BYTES);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        // A: 16 stored values = 32 bytes per step; W: 32 elements = 64 bytes per
-                        // step, steps 2,3 in the second 64-element slice
-                        const uint64_t ad = a_desc + (uint64_t)(j * 2);
-                        const uint64_t bd = b_desc + (uint64_t)((j >> 1) * (Cfg::B_HALF_BYTES >> 4) + (j & 1) * 4);
-                        mma_sp_bf16<CG>(d_tmem, ad, bd, e_tmem + (j & ~1), idesc | (uint32_t)(j & 1),
-                                        (kb > 0 || j > 0) ? 1u : 0u);
-                    }
+                    const uint32_t a_lo = a_lo0 + stage * (Cfg::A_BYTES >> 4);
+                    const uint32_t b_lo = b_lo0 + stage * (Cfg::B_BYTES >> 4);
+                    tmem_cp_128x128b<CG>(e_tmem, e_d0 + (uint64_t)(stage * (Cfg::E_BYTES >> 4)));
+                    // four K steps of 32 logical elements: A advances 32 bytes, W 64 bytes (steps 2, 3
+                    // in the second 64-element slice); metadata column pair + sparse_id2 = step parity
+                    mma_sp_bf16_lh<CG>(d_tmem, a_lo, b_lo, desc_hi, e_tmem, idesc0, accumulate);
+                    mma_sp_bf16_lh<CG>(d_tmem, a_lo + 2, b_lo + 4, desc_hi, e_tmem, idesc1, 1u);
+                    mma_sp_bf16_lh<CG>(d_tmem, a_lo + 4, b_lo + BH, desc_hi, e_tmem + 2, idesc0, 1u);
+                    mma_sp_bf16_lh<CG>(d_tmem, a_lo + 6, b_lo + BH + 4, desc_hi, e_tmem + 2, idesc1, 1u);
+                    accumulate = 1u;
                     if constexpr (CG == 1) tc_commit(bar_empty + 8 * stage);
                     else tc_commit_pair(bar_empty + 8 * stage, 0x3);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
