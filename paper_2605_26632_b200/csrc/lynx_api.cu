@@ -22,6 +22,10 @@ struct lynx_ctx {
     uint32_t* err_dev = nullptr;
     void* scratch = nullptr;  // compressed operands, scale, sums, host staging mirrors
     size_t scratch_bytes = 0;
+    float* sk_partial = nullptr;  // stream-K partial tiles (one slot per cluster) + ready words
+    uint32_t* sk_flags = nullptr;
+    uint32_t sk_epoch = 0;
+    int streamk = 0;  // stream-K tail: off by default (measured: no net gain), LYNX_STREAMK=1 enables
     int64_t launches = 0;
     int gemm_cfg = 0;   // 0 = auto
     int prune_tpu = 0;  // 0 = auto
@@ -124,6 +128,9 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     p.dev_error = ctx->err_dev;
     p.tiles_m = (int)((M + Cfg::BM * Cfg::CG - 1) / (Cfg::BM * Cfg::CG));
     p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
+    p.sk_partial = nullptr;
+    p.sk_flags = nullptr;
+    p.sk_epoch = 0;
 
     auto kern = sparse_gemm_kernel<Cfg>;
     static bool attr_set = false;  // per instantiation
@@ -134,7 +141,27 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     }
     const int tiles = p.tiles_m * p.tiles_n;
     int clusters = ctx->num_sms / Cfg::CG;
-    if (clusters > tiles) clusters = tiles;
+    {
+        // stream-K tail: worth it when the leftover tiles' K blocks give every cluster a piece of
+        // at least 4 blocks; needs the per-cluster partial slots (allocated once, on first use)
+        const int kblocks = (int)(K / Cfg::BK);
+        const int rem = tiles % clusters;
+        if (ctx->streamk && rem > 0 && (int64_t)rem * kblocks >= 4ll * clusters) {
+            if (!ctx->sk_partial) {
+                const size_t slot = (size_t)128 * 256 * 4, nslots = (size_t)ctx->num_sms;
+                void* buf = nullptr;
+                if (cudaMalloc(&buf, nslots * slot + nslots * 8 * 4) != cudaSuccess) return LYNX_ERR_WORKSPACE;
+                if (cudaMemset(buf, 0, nslots * slot + nslots * 8 * 4) != cudaSuccess) return LYNX_ERR_CUDA;
+                ctx->sk_partial = static_cast<float*>(buf);
+                ctx->sk_flags = reinterpret_cast<uint32_t*>(static_cast<char*>(buf) + nslots * slot);
+            }
+            p.sk_partial = ctx->sk_partial;
+            p.sk_flags = ctx->sk_flags;
+            p.sk_epoch = ++ctx->sk_epoch;
+        } else if (clusters > tiles) {
+            clusters = tiles;
+        }
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(clusters * Cfg::CG));
     cfg.blockDim = dim3(Cfg::THREADS);
@@ -223,6 +250,8 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
     *ctx->err_host = DEV_OK;
     const char* env = getenv("LYNX_GEMM_CFG");  // development override of the tile configuration
     if (env) ctx->gemm_cfg = atoi(env);
+    env = getenv("LYNX_STREAMK");  // 1 turns the stream-K tail on
+    if (env) ctx->streamk = atoi(env);
     env = getenv("LYNX_PRUNE_TPU");  // development override: 128-element K blocks per warp
     if (env) ctx->prune_tpu = atoi(env);
     *out = ctx;
@@ -233,6 +262,7 @@ lynx_status lynx_destroy(lynx_ctx* ctx) {
     if (!ctx) return LYNX_ERR_INVALID_ARG;
     cudaSetDevice(ctx->device);
     if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->sk_partial) cudaFree(ctx->sk_partial);
     if (ctx->err_host) cudaFreeHost(ctx->err_host);
     delete ctx;
     return LYNX_OK;

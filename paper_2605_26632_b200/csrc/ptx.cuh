@@ -85,6 +85,35 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Bounded wait for a global-memory word (written with release semantics by another CTA) to reach
+// `want`.  Same time limit and abort protocol as mbar_wait.
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(uint32_t* p, uint32_t v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool flag_wait(const uint32_t* flag, uint32_t want, volatile uint32_t* cta_abort,
+                                          uint32_t* dev_error) {
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (ld_acquire_gpu(flag) == want) return true;
+        if ((it & 0x3f) == 0x3f) {
+            if (*cta_abort) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) {
+                *cta_abort = 1;
+                atomicExch(dev_error, (uint32_t)DEV_TIMEOUT);
+                __threadfence_system();
+                return false;
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------- TMA ------------
 
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {

@@ -32,6 +32,75 @@ struct GemmParams {
     int64_t ldr;
     uint32_t* dev_error;  // sticky error word (host-visible)
     int tiles_m, tiles_n;
+    // stream-K tail (see TileSchedule): fp32 partial tiles, one slot per cluster, and one ready
+    // word per (slot, epilogue warp of the pair) holding the launch epoch; nullptr = off
+    float* sk_partial;
+    uint32_t* sk_flags;
+    uint32_t sk_epoch;
+};
+
+// Work distribution over C persistent clusters.  The first floor(T/C)*C tiles go round-robin,
+// whole.  The K blocks of the remaining R < C tiles are dealt out evenly ("stream-K" tail):
+// cluster c gets tail blocks [c*R*KB/C, (c+1)*R*KB/C), at most two pieces of two tiles.  A piece
+// that ends at its tile's last K block makes that cluster the tile's owner; every other piece
+// is written out as an fp32 partial tile, and the owner adds the partials of the clusters before
+// it in ascending order (fixed order: reproducible).  A cluster does its partial piece first, so
+// nobody who is waited for ever waits.
+struct WorkItem {
+    int tile, kb0, kb1;
+    int kind;           // 0 whole tile, 1 partial piece (write fp32), 2 owner piece (add partials)
+    int first_contrib;  // owner: clusters first_contrib .. c-1 hold the partials
+};
+struct TileSchedule {
+    int T, C, KB, full, R, total;
+    bool streamk;
+    __device__ TileSchedule(int tiles, int clusters, int kblocks, bool enable)
+        : T(tiles), C(clusters), KB(kblocks) {
+        full = (T / C) * C;
+        R = T - full;
+        total = R * KB;
+        streamk = enable && R > 0;
+        if (!streamk) { full = T; R = 0; total = 0; }
+    }
+    // cluster that holds tail block x
+    __device__ int owner_of(int x) const { return (int)((((long long)x + 1) * C - 1) / total); }
+    // does cluster c hold a piece of the tail?
+    __device__ bool has_tail(int c) const {
+        return streamk && (int)((long long)(c + 1) * total / C) > (int)((long long)c * total / C);
+    }
+    __device__ int count(int c) const {
+        int n = 0;
+        for (int t = c; t < full; t += C) ++n;
+        if (streamk) {
+            const int s = (int)((long long)c * total / C), e = (int)((long long)(c + 1) * total / C);
+            if (e > s) n += ((e - 1) / KB != s / KB) ? 2 : 1;
+        }
+        return n;
+    }
+    __device__ WorkItem get(int c, int i) const {
+        WorkItem w{0, 0, KB, 0, 0};
+        const int nfull = (full - c + C - 1) / C > 0 ? (full - c + C - 1) / C : 0;
+        if (i < nfull) { w.tile = c + i * C; return w; }
+        i -= nfull;
+        const int s = (int)((long long)c * total / C), e = (int)((long long)(c + 1) * total / C);
+        const int tA = s / KB, tB = (e - 1) / KB;
+        // pieces: A = [s, min(e, (tA+1)KB)) of tile tA, B = [tB*KB, e) of tile tB (if tB != tA)
+        int a0 = s - tA * KB, a1 = ((e < (tA + 1) * KB) ? e : (tA + 1) * KB) - tA * KB;
+        int b0 = 0, b1 = e - tB * KB;
+        const bool two = tB != tA;
+        const bool a_partial = a1 != KB;            // does not reach the tile's end
+        const bool b_partial = two && b1 != KB;
+        // order: partial piece first
+        bool take_b;
+        if (!two) take_b = false;
+        else take_b = (i == 0) ? (b_partial && !a_partial) : !(b_partial && !a_partial);
+        if (take_b) { w.tile = full + tB; w.kb0 = b0; w.kb1 = b1; }
+        else { w.tile = full + tA; w.kb0 = a0; w.kb1 = a1; }
+        if (w.kb1 != KB) w.kind = 1;
+        else if (w.kb0 != 0) { w.kind = 2; w.first_contrib = owner_of((w.tile - full) * KB); }
+        else w.kind = 0;
+        return w;
+    }
 };
 
 template <int BN_, int CG_, int STAGES_, int CBUFS_>
@@ -97,6 +166,8 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     const int cluster_id = blockIdx.x / CG, num_clusters = gridDim.x / CG;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int kblocks = (int)(p.K / Cfg::BK);
+    const TileSchedule sched(num_tiles, num_clusters, kblocks, p.sk_partial != nullptr);
+    const int num_items = sched.count(cluster_id);
 
     if (threadIdx.x == 0) {
         *cta_abort = 0;
@@ -131,12 +202,13 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             uint32_t issued = 0;
             bool ok = true;
             const uint32_t full0 = (CG == 2) ? mapa(bar_full, 0) : bar_full;  // leader's barriers
-            for (int t = cluster_id; t < num_tiles && ok; t += num_clusters) {
-                const int tm = t % p.tiles_m, tn = t / p.tiles_m;
+            for (int wi = 0; wi < num_items && ok; ++wi) {
+                const WorkItem w = sched.get(cluster_id, wi);
+                const int tm = w.tile % p.tiles_m, tn = w.tile / p.tiles_m;
                 const int m0 = (tm * CG + (int)rank) * Cfg::BM;
                 const int n0 = tn * BN + (int)rank * Cfg::BN_CTA;
                 const int eblk = (tm * CG + (int)rank) * kblocks;
-                for (int kb = 0; kb < kblocks; ++kb) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, cta_abort, p.dev_error)) {
                         ok = false;
                         break;
@@ -180,14 +252,15 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             int it = 0;
-            for (int t = cluster_id; t < num_tiles && ok; t += num_clusters, ++it) {
+            for (; it < num_items && ok; ++it) {
+                const WorkItem w = sched.get(cluster_id, it);
                 const int acc = (Cfg::ACC_STAGES == 2) ? (it & 1) : 0;
                 const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((it >> 1) & 1) : (it & 1);
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, cta_abort, p.dev_error)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 uint32_t accumulate = 0;
-                for (int kb = 0; kb < kblocks; ++kb) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, cta_abort, p.dev_error)) {
                         ok = false;
                         break;
@@ -219,8 +292,10 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         const uint32_t cbuf0 = sC + (warp - 2) * Cfg::CBUFS * Cfg::C_BOX_BYTES;
         const uint32_t tempty0 = (CG == 2) ? mapa(bar_tempty, 0) : bar_tempty;
         int it = 0, cb = 0;
-        for (int t = cluster_id; t < num_tiles; t += num_clusters, ++it) {
-            const int tm = t % p.tiles_m, tn = t / p.tiles_m;
+        bool alive = true;
+        for (; it < num_items && alive; ++it) {
+            const WorkItem w = sched.get(cluster_id, it);
+            const int tm = w.tile % p.tiles_m, tn = w.tile / p.tiles_m;
             const int acc = (Cfg::ACC_STAGES == 2) ? (it & 1) : 0;
             const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((it >> 1) & 1) : (it & 1);
             if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, cta_abort, p.dev_error)) break;
@@ -230,6 +305,23 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             const bool row_ok = row < p.M;
             const float s = (p.row_scale != nullptr && row_ok) ? p.row_scale[row] : 1.0f;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+            // stream-K pieces: this thread's row of the pair tile inside an fp32 partial slot
+            const size_t slot_floats = (size_t)Cfg::BM * CG * BN;
+            // layout of a slot: [64-column chunk][16-byte piece j][row of the pair tile] float4, so a
+            // warp's 32 rows of one piece are 512 contiguous bytes
+            constexpr int SLOT_ROWS = Cfg::BM * CG;
+            const size_t my_row_off = (size_t)((int)rank * Cfg::BM + q * 32 + lane);
+            const int my_flag = (int)rank * 4 + q;
+            if (w.kind == 2) {
+                // wait until every contributing cluster's matching warp has published its rows
+                if (lane == 0) {
+                    for (int cc = w.first_contrib; cc < cluster_id && alive; ++cc)
+                        if (sched.has_tail(cc))
+                            alive = flag_wait(p.sk_flags + cc * 8 + my_flag, p.sk_epoch, cta_abort, p.dev_error);
+                }
+                alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+                if (!alive) break;
+            }
 #pragma unroll 1
             for (int c = 0; c < BN / 64; ++c) {
                 const int n0 = tn * BN + c * 64;
@@ -244,6 +336,35 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     if (lane == 0) {
                         if constexpr (CG == 1) mbar_arrive(bar_tempty + 8 * acc);
                         else mbar_arrive_cluster(tempty0 + 8 * acc);
+                    }
+                }
+                if (w.kind == 1) {
+                    // partial piece: raw fp32 accumulators to this cluster's slot
+                    float4* dst = reinterpret_cast<float4*>(p.sk_partial + (size_t)cluster_id * slot_floats) +
+                                  (size_t)c * 16 * SLOT_ROWS + my_row_off;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        __stcg(dst + (size_t)j * SLOT_ROWS, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                    __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+                    continue;
+                }
+                if (w.kind == 2) {
+                    // owner piece: add the partials in ascending cluster order
+                    for (int cc = w.first_contrib; cc < cluster_id; ++cc) {
+                        if (!sched.has_tail(cc)) continue;
+                        const float4* src = reinterpret_cast<const float4*>(p.sk_partial + (size_t)cc * slot_floats) +
+                                            (size_t)c * 16 * SLOT_ROWS + my_row_off;
+                        float4 pa[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) pa[j] = __ldcg(src + (size_t)j * SLOT_ROWS);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float4 a = pa[j];
+                            v[4 * j] = __float_as_uint(__uint_as_float(v[4 * j]) + a.x);
+                            v[4 * j + 1] = __float_as_uint(__uint_as_float(v[4 * j + 1]) + a.y);
+                            v[4 * j + 2] = __float_as_uint(__uint_as_float(v[4 * j + 2]) + a.z);
+                            v[4 * j + 3] = __float_as_uint(__uint_as_float(v[4 * j + 3]) + a.w);
+                        }
                     }
                 }
                 if (n0 >= p.N) continue;
@@ -289,6 +410,12 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     tma_store_commit();
                 }
                 cb = (cb + 1 == Cfg::CBUFS) ? 0 : cb + 1;
+            }
+            if (w.kind == 1) {
+                // publish: all lanes' stores, then the ready word of this (slot, warp)
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) st_release_gpu(p.sk_flags + cluster_id * 8 + my_flag, p.sk_epoch);
             }
         }
         if (lane == 0) tma_store_wait_all<0>();

@@ -184,6 +184,31 @@ def test_every_tile_configuration(cfg, monkeypatch):
         ctx.close()
 
 
+@pytest.mark.parametrize("cfg", [4, 5])
+def test_stream_k_tail_matches_oracle_and_is_deterministic(cfg, monkeypatch):
+    """Optional stream-K tail (leftover tiles split along K, fp32 partial tiles added in fixed
+    order): same answer within tolerance, bit-identical run to run."""
+    from paper_2605_26632_b200 import binding
+
+    monkeypatch.setenv("LYNX_GEMM_CFG", str(cfg))
+    monkeypatch.setenv("LYNX_STREAMK", "1")
+    ctx = binding.Lynx(0)
+    try:
+        wl = inputs.Workload("t", 2304, 2048, 2304, "outlier", 55)  # 81 / 108 tiles on 74 CTA pairs
+        d = inputs.make_workload(wl, with_bias=True)
+        X, W, b = d["X"].cuda(), d["W"].cuda(), d["bias"].cuda()
+        rows = np.arange(0, wl.M, 37, dtype=np.int64)
+        ref = oracle.act_sparse_linear(u16(X), u16(W), bias=u16(b), comp_mode=1, rows=rows)
+        Y1 = ctx.act_sparse_linear(X, W, b, 1)
+        Y2 = ctx.act_sparse_linear(X, W, b, 1)
+        check_y(Y1[torch.from_numpy(rows).cuda()], ref["Y"])
+        assert torch.equal(Y1, Y2)
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
+
+
 @pytest.mark.parametrize("M,K,N", [(1, 128, 8), (5, 256, 72), (129, 384, 200), (257, 128, 1000)])
 def test_ragged_shapes(lx, M, K, N):
     wl = inputs.Workload("t", M, K, N, "normal", 31)
