@@ -12,6 +12,7 @@
 
 #include "prune_compress.cuh"
 #include "sparse_gemm.cuh"
+#include "fused_linear.cuh"
 
 using namespace lynx;
 
@@ -203,6 +204,43 @@ lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int
 #undef LYNX_GEMM_ARGS
 }
 
+// One-kernel path: raw X is pruned inside the GEMM kernel.
+lynx_status launch_fused(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, const void* W, int64_t N,
+                         int64_t ldw, const void* bias, int with_scale, const void* residual, int64_t ldr, void* Y,
+                         int64_t ldy, cudaStream_t st) {
+    using Cfg = FusedCfg;
+    CUtensorMap tx, tb, ty;
+    if (!make_tmap_2d(&tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx * 2, 64,
+                      Cfg::BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)N, (uint64_t)K, (uint64_t)ldw * 2, 64,
+                      Cfg::BN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, 64,
+                      32, CU_TENSOR_MAP_SWIZZLE_128B))
+        return LYNX_ERR_CUDA;
+    FusedParams p;
+    p.M = M; p.N = N; p.K = K;
+    p.with_scale = with_scale;
+    p.bias = static_cast<const uint16_t*>(bias);
+    p.residual = static_cast<const uint16_t*>(residual);
+    p.ldr = ldr;
+    p.dev_error = ctx->err_dev;
+    p.tiles_m = (int)((M + Cfg::BM - 1) / Cfg::BM);
+    p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(fused_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Cfg::SMEM_BYTES) != cudaSuccess)
+            return LYNX_ERR_CUDA;
+        attr_set = true;
+    }
+    int grid = p.tiles_m * p.tiles_n;
+    if (grid > ctx->num_sms) grid = ctx->num_sms;
+    fused_linear_kernel<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, st>>>(tx, tb, ty, p);
+    if (cudaGetLastError() != cudaSuccess) return LYNX_ERR_CUDA;
+    ctx->launches++;
+    return LYNX_OK;
+}
+
 lynx_status check_common(lynx_ctx* ctx, int64_t M, int64_t K) {
     if (!ctx) return LYNX_ERR_INVALID_ARG;
     if (M < 1 || K < 128) return LYNX_ERR_INVALID_ARG;
@@ -385,8 +423,21 @@ lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int6
     lynx_status s = check_common(ctx, M, K);
     if (s != LYNX_OK) return s;
     if (fuse != LYNX_FUSE_AUTO && fuse != LYNX_FUSE_SEPARATE && fuse != LYNX_FUSE_FUSED) return LYNX_ERR_INVALID_ARG;
-    if (fuse == LYNX_FUSE_FUSED) return LYNX_ERR_UNSUPPORTED_SHAPE;  // fused kernel: not built yet
     if (N < 8) return LYNX_ERR_INVALID_ARG;
+    if (fuse == LYNX_FUSE_FUSED) {
+        // the whole-tensor scale needs all of X before the first output: two-kernel path only
+        if (mode == LYNX_COMP_TENSOR) return LYNX_ERR_UNSUPPORTED_SHAPE;
+        if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW) return LYNX_ERR_INVALID_ARG;
+        if (!X || !W || !Y) return LYNX_ERR_INVALID_ARG;
+        if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
+        if (ldx < K || ldw < K || ldy < N || (residual && ldr < N)) return LYNX_ERR_INVALID_ARG;
+        if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || (ldx % 8) || (ldw % 8) || (ldy % 8) ||
+            (bias && !aligned16(bias)) || (residual && (!aligned16(residual) || (ldr % 8))))
+            return LYNX_ERR_ALIGNMENT;
+        if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+        return launch_fused(ctx, X, M, K, ldx, W, N, ldw, bias, mode == LYNX_COMP_ROW ? 1 : 0, residual, ldr, Y, ldy,
+                            static_cast<cudaStream_t>(stream));
+    }
     ScratchLayout L = scratch_layout(M, N, K);
     {
         std::lock_guard<std::mutex> lock(ctx->mu);

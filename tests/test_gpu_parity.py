@@ -264,6 +264,78 @@ def test_host_buffer_entry_point(lx):
     check_y(Y, ref["Y"])
 
 
+# ------------------------------------------------------------------ fused one-kernel path ------
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("with_bias,with_res", [(False, False), (True, True)])
+def test_fused_tiny_config_full_oracle(lx, mode, with_bias, with_res):
+    from paper_2605_26632_b200 import binding
+
+    wl = inputs.WORKLOADS["tiny"]
+    d = inputs.make_workload(wl, with_bias=with_bias, with_residual=with_res)
+    X, W = d["X"].cuda(), d["W"].cuda()
+    b = d["bias"].cuda() if with_bias else None
+    r = d["residual"].cuda() if with_res else None
+    ref = oracle.act_sparse_linear(u16(X), u16(W), bias=None if b is None else u16(b), comp_mode=mode,
+                                   Yr=None if r is None else u16(r))
+    Yf = lx.act_sparse_linear(X, W, b, mode, r, fuse=binding.FUSE_FUSED)
+    check_y(Yf, ref["Y"])
+    if mode == 0:
+        # same products in the same order as the two-kernel path: identical bits
+        Ys = lx.act_sparse_linear(X, W, b, mode, r, fuse=binding.FUSE_SEPARATE)
+        assert torch.equal(Yf, Ys)
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 128, 8), (129, 384, 200), (300, 640, 456), (520, 1024, 1000)])
+def test_fused_ragged_shapes(lx, M, K, N):
+    from paper_2605_26632_b200 import binding
+
+    wl = inputs.Workload("t", M, K, N, "outlier", 61)
+    d = inputs.make_workload(wl, with_bias=True, with_residual=True)
+    X, W, b, r = d["X"].cuda(), d["W"].cuda(), d["bias"].cuda(), d["residual"].cuda()
+    ref = oracle.act_sparse_linear(u16(X), u16(W), bias=u16(b), comp_mode=1, Yr=u16(r))
+    Y = lx.act_sparse_linear(X, W, b, 1, r, fuse=binding.FUSE_FUSED)
+    check_y(Y, ref["Y"])
+    Y2 = lx.act_sparse_linear(X, W, b, 1, r, fuse=binding.FUSE_FUSED)
+    assert torch.equal(Y, Y2)
+
+
+def test_fused_identity_weight_and_special_values(lx):
+    """W = I through the fused kernel: its in-kernel selection, value packing and metadata must
+    reproduce mask * X exactly, including NaN / Inf / subnormal ranking."""
+    from paper_2605_26632_b200 import binding
+
+    M, K = 200, 512
+    X = inputs.make_x(M, K, "normal", 13).cuda()
+    W = torch.eye(K, dtype=torch.bfloat16, device="cuda")
+    Y = lx.act_sparse_linear(X, W, None, 0, None, fuse=binding.FUSE_FUSED)
+    Xu = u16(X)
+    want = oracle.bf16_to_f32(Xu * oracle.topk24_mask(Xu))
+    assert (Y.float().cpu().numpy() == want).all()
+
+
+def test_fused_full_size_mlp_up(lx):
+    from paper_2605_26632_b200 import binding
+
+    wl = inputs.WORKLOADS["mlp_up"]
+    d = inputs.make_workload(wl, with_bias=True)
+    X, W, b = d["X"].cuda(), d["W"].cuda(), d["bias"].cuda()
+    Y = lx.act_sparse_linear(X, W, b, 1, None, fuse=binding.FUSE_FUSED)
+    rows = np.sort(np.random.default_rng(4).choice(wl.M, 24, replace=False)).astype(np.int64)
+    ref = oracle.act_sparse_linear(u16(d["X"]), u16(d["W"]), bias=u16(d["bias"]), comp_mode=1, rows=rows)
+    check_y(Y[torch.from_numpy(rows).cuda()], ref["Y"])
+
+
+def test_fused_rejects_whole_tensor_scale(lx):
+    from paper_2605_26632_b200 import binding
+
+    X = torch.zeros(16, 128, dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros(16, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.LynxError) as e:
+        lx.act_sparse_linear(X, W, None, 2, None, fuse=binding.FUSE_FUSED)
+    assert e.value.status == 2
+
+
 # ------------------------------------------------------------------ full-size workloads --------
 
 def _full_size_case(lx, wl, n_rows, mode=1):
