@@ -28,6 +28,7 @@ struct lynx_ctx {
     uint32_t sk_epoch = 0;
     int streamk = 0;  // stream-K tail: off by default (measured: no net gain), LYNX_STREAMK=1 enables
     int64_t launches = 0;
+    int pdl = 1;        // programmatic dependent launch of the finalize and GEMM kernels
     int gemm_cfg = 0;   // 0 = auto
     int prune_tpu = 0;  // 0 = auto
     std::mutex mu;
@@ -168,13 +169,16 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     cfg.blockDim = dim3(Cfg::THREADS);
     cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = Cfg::CG;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // let the prologue (barriers, tensor memory, descriptor prefetch) overlap the previous kernel
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, te, ty, p);
     if (e != cudaSuccess) return LYNX_ERR_CUDA;
     ctx->launches++;
@@ -186,10 +190,20 @@ lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int
                         cudaStream_t st) {
     int cfg = ctx->gemm_cfg;
     if (cfg == 0) {
-        // CTA-pair tiles.  Long K amortises the epilogue, so the single-accumulator 256 x 256 tile
-        // (fewest operand bytes per flop) wins; short K needs the epilogue hidden behind the next
-        // tile's main loop, which the double-buffered 256 x 192 tile provides.
-        cfg = (K >= 6144) ? 5 : 4;
+        // CTA-pair tiles 256 x {256, 192, 128}.  Pick the one with the smallest modelled time:
+        // rounds of tiles over the CTA pairs x (K blocks x measured time per K block + exposed
+        // epilogue).  Per-K-block times (us) are measured B200 figures for each tile shape; the
+        // 256-wide tile has one accumulator buffer, so its epilogue is not hidden.
+        const int pairs = ctx->num_sms / 2;
+        const double kb = (double)(K / 128);
+        struct { int id, bn; double t_kb, epi; } cand[3] = {{5, 256, 0.50, 3.0}, {4, 192, 0.415, 0.6}, {6, 128, 0.345, 0.5}};
+        double best = 1e30;
+        for (auto& c : cand) {
+            const int64_t tiles = ((M + 255) / 256) * ((N + c.bn - 1) / c.bn);
+            const double rounds = (double)((tiles + pairs - 1) / pairs);
+            const double t = rounds * (kb * c.t_kb + c.epi);
+            if (t < best) { best = t; cfg = c.id; }
+        }
     }
 #define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, Y, ldy, st
     switch (cfg) {
@@ -288,6 +302,8 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
     *ctx->err_host = DEV_OK;
     const char* env = getenv("LYNX_GEMM_CFG");  // development override of the tile configuration
     if (env) ctx->gemm_cfg = atoi(env);
+    env = getenv("LYNX_PDL");  // 0 turns programmatic dependent launch off
+    if (env) ctx->pdl = atoi(env);
     env = getenv("LYNX_STREAMK");  // 1 turns the stream-K tail on
     if (env) ctx->streamk = atoi(env);
     env = getenv("LYNX_PRUNE_TPU");  // development override: 128-element K blocks per warp
@@ -377,17 +393,43 @@ lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t
     }
     const int64_t units = rb16 * KS;
     const unsigned grid = (unsigned)((units + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS);
-    if (mode == LYNX_COMP_NONE)
-        prune_compress_kernel<false><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
-            static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
-            row_scale, nullptr, nullptr, 0, tpu, KS, units);
-    else
-        prune_compress_kernel<true><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
-            static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
-            row_scale, sums, partial, (int)mode, tpu, KS, units);
+    {
+        cudaLaunchConfig_t pc = {};
+        pc.gridDim = dim3(grid);
+        pc.blockDim = dim3(PRUNE_CTA_WARPS * 32);
+        pc.stream = st;
+        cudaLaunchAttribute pa[1];
+        pa[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        pa[0].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
+        pc.attrs = pa;
+        pc.numAttrs = 1;
+        const uint16_t* Xp = static_cast<const uint16_t*>(X);
+        uint16_t* vp = static_cast<uint16_t*>(values);
+        uint8_t* mp = static_cast<uint8_t*>(meta);
+        float* none_f = nullptr;
+        cudaError_t e;
+        if (mode == LYNX_COMP_NONE)
+            e = cudaLaunchKernelEx(&pc, prune_compress_kernel<false>, Xp, M, K, ldx, vp, mp, row_scale, none_f, none_f,
+                                   0, tpu, KS, units);
+        else
+            e = cudaLaunchKernelEx(&pc, prune_compress_kernel<true>, Xp, M, K, ldx, vp, mp, row_scale, sums, partial,
+                                   (int)mode, tpu, KS, units);
+        if (e != cudaSuccess) return LYNX_ERR_CUDA;
+    }
     ctx->launches++;
     if (mode != LYNX_COMP_NONE && KS > 1) {
-        row_scale_kernel<<<(unsigned)((M + 15) / 16), 256, 0, st>>>(partial, M, KS, (int)mode, row_scale, sums);
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3((unsigned)((M + 15) / 16));
+        lc.blockDim = dim3(256);
+        lc.stream = st;
+        cudaLaunchAttribute la[1];
+        la[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        la[0].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
+        lc.attrs = la;
+        lc.numAttrs = 1;
+        const float* partial_c = partial;
+        if (cudaLaunchKernelEx(&lc, row_scale_kernel, partial_c, M, KS, (int)mode, row_scale, sums) != cudaSuccess)
+            return LYNX_ERR_CUDA;
         ctx->launches++;
     }
     if (mode == LYNX_COMP_TENSOR) {

@@ -175,6 +175,7 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid < 64) lut[tid] = prune_lut_entry(tid & 15, tid >> 4);
     __syncthreads();
+    griddep_wait();  // no-op unless launched as a programmatic dependent of the previous kernel
 
     const int64_t unit = (int64_t)blockIdx.x * PRUNE_CTA_WARPS + warp;
     if (unit >= num_units) return;
@@ -235,6 +236,7 @@ __global__ void __launch_bounds__(256)
 row_scale_kernel(const float* __restrict__ partial, int64_t M, int KS, int mode, float* __restrict__ row_scale,
                  float* __restrict__ sums) {
     __shared__ float2 red[16][16];
+    griddep_wait();  // launched early (programmatic dependent launch): partial sums must be complete
     const int row = threadIdx.x & 15, jl = threadIdx.x >> 4;
     const int64_t rb16 = blockIdx.x;
     const float2* p = reinterpret_cast<const float2*>(partial) + rb16 * KS * 16 + row;

@@ -164,6 +164,11 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// Programmatic dependent launch: a kernel launched with the "programmatic stream serialization"
+// attribute may start while its predecessor in the stream is still draining; it must execute this
+// wait before it touches anything the predecessor wrote (or still reads).
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------------------- cluster --------
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {

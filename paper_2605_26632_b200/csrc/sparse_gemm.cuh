@@ -194,6 +194,8 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     if constexpr (CG == 2) cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above overlapped the previous kernel's tail; its results are needed from here on
+    griddep_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer ----------

@@ -1,0 +1,81 @@
+"""Times every stage of the path over the DiT shape sweep and prints a markdown table.
+
+    python -m paper_2605_26632_b200.sweep [--quick] [--iters 30]
+
+For each (M, K, N): prune/compress alone (GB/s of its 3.125 B/element), sparse GEMM alone, the
+two-kernel layer, the fused one-kernel layer, and the dense bf16 linear (torch / cuBLASLt) on the
+same GPU with the same timing loop.  Inputs rotate over enough copies that nothing a launch reads
+is left in the L2 by the previous launch; times are CUDA-event averages over `iters` launches.
+"""
+from __future__ import annotations
+
+import argparse
+import math
+
+import torch
+
+from . import binding, inputs
+
+
+def timeloop(fn, nsets, iters, warm=5):
+    for i in range(warm):
+        fn(i % nsets)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(iters):
+        fn(i % nsets)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / iters  # ms
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--quick", action="store_true", help="M = 4096 only")
+    ap.add_argument("--iters", type=int, default=30)
+    ap.add_argument("--no-fused", action="store_true")
+    args = ap.parse_args()
+    lx = binding.Lynx(0)
+    Ms = (4096,) if args.quick else inputs.SWEEP_M
+    shapes = [(M, K, N) for M in Ms for (K, N) in inputs.SWEEP_KN]
+    shapes += [(4352, 3072, 9216), (4352, 3072, 3072)]
+    if not args.quick:
+        shapes += [(M, K, M) for M in (2048, 4096, 8192) for K in (3072, 12288)]  # the paper's kernel grid
+    print("| M | K | N | prune us | prune GB/s | GEMM us | GEMM TF | layer us | layer TF | fused us | fused TF | "
+          "dense us | dense TF | GEMM/dense | layer/dense |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for (M, K, N) in shapes:
+        per_set = M * K * 2 + M * K + M * K // 8 + N * K * 2 + M * N * 2
+        nsets = max(2, math.ceil(400e6 / per_set))
+        g = torch.Generator(device="cuda").manual_seed(M + K + N)
+        Xs = [torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16) for _ in range(nsets)]
+        Ws = [(torch.randn(N, K, device="cuda", generator=g) * K ** -0.5).to(torch.bfloat16) for _ in range(nsets)]
+        b = torch.zeros(N, device="cuda", dtype=torch.bfloat16)
+        vs = [torch.empty(M, K // 2, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+        ms = [torch.empty(binding.meta_bytes(M, K), device="cuda", dtype=torch.uint8) for _ in range(nsets)]
+        ss = [torch.empty(M, device="cuda", dtype=torch.float32) for _ in range(nsets)]
+        Ys = [torch.empty(M, N, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+        lx.reserve(M, N, K)
+        for j in range(nsets):
+            lx.prune_compress(Xs[j], 1, vs[j], ms[j], ss[j])
+        it = args.iters
+        tp = timeloop(lambda j: lx.prune_compress(Xs[j], 1, vs[j], ms[j], ss[j]), nsets, it)
+        tg = timeloop(lambda j: lx.sparse_linear(vs[j], ms[j], Ws[j], b, ss[j], None, Ys[j]), nsets, it)
+        tl = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_SEPARATE), nsets, it)
+        tf = float("nan")
+        if not args.no_fused:
+            tf = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_FUSED), nsets, it)
+        td = timeloop(lambda j: torch.nn.functional.linear(Xs[j], Ws[j], b), nsets, it)
+        fl = 2.0 * M * N * K
+        tf_s = lambda t: fl / t / 1e9
+        print(f"| {M} | {K} | {N} | {tp*1e3:.1f} | {M*K*3.125/tp/1e6:.0f} | {tg*1e3:.1f} | {tf_s(tg):.0f} | "
+              f"{tl*1e3:.1f} | {tf_s(tl):.0f} | {tf*1e3:.1f} | {tf_s(tf):.0f} | {td*1e3:.1f} | {tf_s(td):.0f} | "
+              f"{td/tg:.2f} | {td/tl:.2f} |", flush=True)
+        assert lx.last_error() == 0
+        del Xs, Ws, vs, ms, ss, Ys
+        torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    main()
