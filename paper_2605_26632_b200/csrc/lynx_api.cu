@@ -23,6 +23,7 @@ struct lynx_ctx {
     uint32_t* err_dev = nullptr;
     void* scratch = nullptr;  // compressed operands, scale, sums, host staging mirrors
     size_t scratch_bytes = 0;
+    uint32_t* tickets = nullptr;  // one word per 16-row block (prune finalize), zero between launches
     float* sk_partial = nullptr;  // stream-K partial tiles (one slot per cluster) + ready words
     uint32_t* sk_flags = nullptr;
     uint32_t sk_epoch = 0;
@@ -79,6 +80,8 @@ lynx_status check_device_error(lynx_ctx* ctx) {
 lynx_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? LYNX_OK : LYNX_ERR_CUDA; }
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+constexpr size_t PRUNE_TICKET_BYTES = 1u << 20;  // 262144 row blocks of 16 rows = 4M rows
 
 // Scratch layout for (M, N, K):
 // [partial row sums][sums 2M floats][values][meta][row_scale M floats][X stage][Y stage]
@@ -300,6 +303,12 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
         return LYNX_ERR_CUDA;
     }
     *ctx->err_host = DEV_OK;
+    if (cudaMalloc(reinterpret_cast<void**>(&ctx->tickets), PRUNE_TICKET_BYTES) != cudaSuccess ||
+        cudaMemset(ctx->tickets, 0, PRUNE_TICKET_BYTES) != cudaSuccess) {
+        cudaFreeHost(ctx->err_host);
+        delete ctx;
+        return LYNX_ERR_WORKSPACE;
+    }
     const char* env = getenv("LYNX_GEMM_CFG");  // development override of the tile configuration
     if (env) ctx->gemm_cfg = atoi(env);
     env = getenv("LYNX_PDL");  // 0 turns programmatic dependent launch off
@@ -317,6 +326,7 @@ lynx_status lynx_destroy(lynx_ctx* ctx) {
     cudaSetDevice(ctx->device);
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->sk_partial) cudaFree(ctx->sk_partial);
+    if (ctx->tickets) cudaFree(ctx->tickets);
     if (ctx->err_host) cudaFreeHost(ctx->err_host);
     delete ctx;
     return LYNX_OK;
@@ -391,8 +401,9 @@ lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t
         partial = reinterpret_cast<float*>(base + L.partial);
         sums = reinterpret_cast<float*>(base + L.sums);
     }
-    const int64_t units = rb16 * KS;
-    const unsigned grid = (unsigned)((units + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS);
+    if ((size_t)rb16 * 4 > PRUNE_TICKET_BYTES) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    const int ctas_per_rb = (KS + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS;
+    const unsigned grid = (unsigned)(rb16 * ctas_per_rb);
     {
         cudaLaunchConfig_t pc = {};
         pc.gridDim = dim3(grid);
@@ -407,31 +418,17 @@ lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t
         uint16_t* vp = static_cast<uint16_t*>(values);
         uint8_t* mp = static_cast<uint8_t*>(meta);
         float* none_f = nullptr;
+        uint32_t* none_u = nullptr;
         cudaError_t e;
         if (mode == LYNX_COMP_NONE)
             e = cudaLaunchKernelEx(&pc, prune_compress_kernel<false>, Xp, M, K, ldx, vp, mp, row_scale, none_f, none_f,
-                                   0, tpu, KS, units);
+                                   none_u, 0, tpu, KS, ctas_per_rb);
         else
             e = cudaLaunchKernelEx(&pc, prune_compress_kernel<true>, Xp, M, K, ldx, vp, mp, row_scale, sums, partial,
-                                   (int)mode, tpu, KS, units);
+                                   ctx->tickets, (int)mode, tpu, KS, ctas_per_rb);
         if (e != cudaSuccess) return LYNX_ERR_CUDA;
     }
     ctx->launches++;
-    if (mode != LYNX_COMP_NONE && KS > 1) {
-        cudaLaunchConfig_t lc = {};
-        lc.gridDim = dim3((unsigned)((M + 15) / 16));
-        lc.blockDim = dim3(256);
-        lc.stream = st;
-        cudaLaunchAttribute la[1];
-        la[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        la[0].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
-        lc.attrs = la;
-        lc.numAttrs = 1;
-        const float* partial_c = partial;
-        if (cudaLaunchKernelEx(&lc, row_scale_kernel, partial_c, M, KS, (int)mode, row_scale, sums) != cudaSuccess)
-            return LYNX_ERR_CUDA;
-        ctx->launches++;
-    }
     if (mode == LYNX_COMP_TENSOR) {
         tensor_scale_kernel<<<1, 1024, 0, st>>>(sums, M, row_scale);
         ctx->launches++;
@@ -606,26 +603,28 @@ extern "C" lynx_status lynx_prune_compress_static(const void* X, int64_t M, int6
     int tpu = (int)(want < 1 ? 1 : (want > 8 ? 8 : want));
     while (kblocks % tpu) --tpu;
     const int KS = (int)(kblocks / tpu);
-    // static scratch: [partial sums: rb16 * KS * 32 floats][per-row sums: 2 * M floats]
+    // static scratch: [tickets: 64 KB][partial sums: rb16 * KS * 32 floats][per-row sums: 2 * M floats]
+    // (a __device__ array starts zeroed and every launch leaves its tickets at zero again)
+    constexpr size_t STATIC_TICKET_BYTES = 64u << 10;
+    if ((size_t)rb16 * 4 > STATIC_TICKET_BYTES) return LYNX_ERR_WORKSPACE;
     const size_t partial_bytes = (mode != LYNX_COMP_NONE && KS > 1) ? (size_t)rb16 * KS * 32 * 4 : 0;
     const size_t partial_padded = (partial_bytes + 255) / 256 * 256;
     const size_t sums_bytes = (mode == LYNX_COMP_TENSOR) ? (size_t)M * 8 : 0;
-    if (partial_padded + sums_bytes > (size_t)LYNX_STATIC_SCRATCH_BYTES) return LYNX_ERR_WORKSPACE;
-    float* partial = reinterpret_cast<float*>(scratch);
-    float* sums = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + partial_padded);
+    if (STATIC_TICKET_BYTES + partial_padded + sums_bytes > (size_t)LYNX_STATIC_SCRATCH_BYTES) return LYNX_ERR_WORKSPACE;
+    uint32_t* tickets = reinterpret_cast<uint32_t*>(scratch);
+    float* partial = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + STATIC_TICKET_BYTES);
+    float* sums = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + STATIC_TICKET_BYTES + partial_padded);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int64_t units = rb16 * KS;
-    const unsigned grid = (unsigned)((units + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS);
+    const int ctas_per_rb = (KS + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS;
+    const unsigned grid = (unsigned)(rb16 * ctas_per_rb);
     if (mode == LYNX_COMP_NONE)
         prune_compress_kernel<false><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
             static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
-            row_scale, nullptr, nullptr, 0, tpu, KS, units);
+            row_scale, nullptr, nullptr, nullptr, 0, tpu, KS, ctas_per_rb);
     else
         prune_compress_kernel<true><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
             static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
-            row_scale, sums, partial, (int)mode, tpu, KS, units);
-    if (mode != LYNX_COMP_NONE && KS > 1)
-        row_scale_kernel<<<(unsigned)((M + 15) / 16), 256, 0, st>>>(partial, M, KS, (int)mode, row_scale, sums);
+            row_scale, sums, partial, tickets, (int)mode, tpu, KS, ctas_per_rb);
     if (mode == LYNX_COMP_TENSOR) tensor_scale_kernel<<<1, 1024, 0, st>>>(sums, M, row_scale);
     return cuda_ok(cudaGetLastError());
 }

@@ -100,8 +100,8 @@ __device__ __forceinline__ uint32_t prune_vec16(const uint32_t (&r)[8], const ui
 // Work unit of one warp: 16 rows x (tiles_per_unit * 128) elements; the KS = kblocks /
 // tiles_per_unit units of a 16-row block are independent warps (many small CTAs keep the SMs'
 // load queues full).  With KS > 1 each unit writes its partial row sums
-// (partial[(rb16*KS + ks)*32 + 2*row + {0: sum x^2, 1: sum kept x^2}]) and row_scale_kernel adds
-// them in fixed order, so the result does not depend on scheduling.
+// (partial[(rb16*KS + ks)*32 + 2*row + {0: sum x^2, 1: sum kept x^2}]) and the last CTA of the row
+// block to finish adds them in a fixed order, so the result does not depend on scheduling.
 //
 // mode: 0 none (row_scale written as 1 if non-null), 1 per-row scale, 2 per-row sums for the
 // whole-tensor scale (sums[2*m] = sum x^2, sums[2*m+1] = sum kept x^2).
@@ -113,10 +113,16 @@ __device__ __forceinline__ uint32_t prune_vec16(const uint32_t (&r)[8], const ui
 #endif
 constexpr int PRUNE_CTA_WARPS = LYNX_PRUNE_CTA_WARPS;
 
+// Results of one 16 x 128 tile held in registers until they are stored.
+struct TileOut {
+    uint32_t oa[8], ob[8];  // 16 kept values of row r / row r + 8
+    uint32_t w0, w1;        // the lane's two metadata words
+};
+
 template <bool SUMS, bool GUARD>
-__device__ __forceinline__ void prune_tile(const uint16_t* xa, const uint16_t* xb, uint16_t* va, uint16_t* vb,
-                                           uint32_t* slab, bool okA, bool okB, const uint32_t* lut, float& numA,
-                                           float& denA, float& numB, float& denB) {
+__device__ __forceinline__ void prune_tile_compute(const uint16_t* xa, const uint16_t* xb, bool okA, bool okB,
+                                                   const uint32_t* lut, TileOut& out, float& numA, float& denA,
+                                                   float& numB, float& denB) {
     uint32_t a0[8], a1[8], b0[8], b1[8];
     if constexpr (GUARD) {
 #pragma unroll
@@ -135,16 +141,13 @@ __device__ __forceinline__ void prune_tile(const uint16_t* xa, const uint16_t* x
         ldg256_stream(xb, b0);
         ldg256_stream(xb + 16, b1);
     }
-    uint32_t oa[8], ob[8];
-    const uint32_t ma0 = prune_vec16(a0, lut, oa);
-    const uint32_t ma1 = prune_vec16(a1, lut, oa + 4);
-    const uint32_t mb0 = prune_vec16(b0, lut, ob);
-    const uint32_t mb1 = prune_vec16(b1, lut, ob + 4);
-    if (!GUARD || okA) stg256(va, oa);
-    if (!GUARD || okB) stg256(vb, ob);
+    const uint32_t ma0 = prune_vec16(a0, lut, out.oa);
+    const uint32_t ma1 = prune_vec16(a1, lut, out.oa + 4);
+    const uint32_t mb0 = prune_vec16(b0, lut, out.ob);
+    const uint32_t mb1 = prune_vec16(b1, lut, out.ob + 4);
     // rows past M prune to the pattern (0,1) = nibble 0x4, the documented padding
-    slab[0] = ma0 | (mb0 << 16);
-    slab[32] = ma1 | (mb1 << 16);
+    out.w0 = ma0 | (mb0 << 16);
+    out.w1 = ma1 | (mb1 << 16);
     if constexpr (SUMS) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -158,10 +161,18 @@ __device__ __forceinline__ void prune_tile(const uint16_t* xa, const uint16_t* x
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            denA = fma_sq_bf16x2(oa[i], denA);
-            denB = fma_sq_bf16x2(ob[i], denB);
+            denA = fma_sq_bf16x2(out.oa[i], denA);
+            denB = fma_sq_bf16x2(out.ob[i], denB);
         }
     }
+}
+
+__device__ __forceinline__ void prune_tile_store(const TileOut& out, uint16_t* va, uint16_t* vb, uint32_t* slab,
+                                                 bool okA, bool okB) {
+    if (okA) stg256(va, out.oa);
+    if (okB) stg256(vb, out.ob);
+    slab[0] = out.w0;
+    slab[32] = out.w1;
 }
 
 template <bool SUMS>
@@ -169,41 +180,51 @@ __global__ void __launch_bounds__(PRUNE_CTA_WARPS * 32, LYNX_PRUNE_MIN_CTAS)
 prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int64_t ldx,
                       uint16_t* __restrict__ values, uint8_t* __restrict__ meta,
                       float* __restrict__ row_scale, float* __restrict__ sums,
-                      float* __restrict__ partial, int mode, int tiles_per_unit, int KS,
-                      int64_t num_units) {
+                      float* __restrict__ partial, uint32_t* __restrict__ tickets, int mode,
+                      int tiles_per_unit, int KS, int ctas_per_rb) {
     __shared__ uint32_t lut[4 * 16];
+    __shared__ float2 red[PRUNE_CTA_WARPS * 2][16];
+    __shared__ uint32_t s_last;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid < 64) lut[tid] = prune_lut_entry(tid & 15, tid >> 4);
     __syncthreads();
     griddep_wait();  // no-op unless launched as a programmatic dependent of the previous kernel
 
-    const int64_t unit = (int64_t)blockIdx.x * PRUNE_CTA_WARPS + warp;
-    if (unit >= num_units) return;
-    const int64_t rb16 = unit / KS;
-    const int ks = (int)(unit - rb16 * KS);
+    // CTA -> 16-row block and its first K unit; the CTAs of a row block are consecutive
+    const int64_t rb16 = blockIdx.x / ctas_per_rb;
+    const int ks = (int)(blockIdx.x % ctas_per_rb) * PRUNE_CTA_WARPS + warp;
+    const bool active = ks < KS;
     const int64_t row0 = rb16 * PRUNE_ROWS;
     const int r = lane >> 2, q = lane & 3;
     const int64_t rowA = row0 + r, rowB = rowA + 8;
     const int64_t kblocks = K / 128;
-    const int64_t kb0 = (int64_t)ks * tiles_per_unit;
-    // metadata slab of this row block inside block (row0/128, kb)
-    uint32_t* slab = reinterpret_cast<uint32_t*>(meta + ((row0 / 128) * kblocks + kb0) * 2048 +
-                                                 ((row0 % 128) / 16) * 256 + lane * 4);
-    const uint16_t* xa = X + rowA * ldx + kb0 * 128 + q * 32;
-    const uint16_t* xb = xa + 8 * ldx;
-    uint16_t* va = values + rowA * (K / 2) + kb0 * 64 + q * 16;
-    uint16_t* vb = va + 8 * (K / 2);
-
     float numA = 0.f, denA = 0.f, numB = 0.f, denB = 0.f;
-    if (row0 + PRUNE_ROWS <= M) {
-        for (int t = 0; t < tiles_per_unit; ++t)
-            prune_tile<SUMS, false>(xa + t * 128, xb + t * 128, va + t * 64, vb + t * 64, slab + t * 512, true,
-                                    true, lut, numA, denA, numB, denB);
-    } else {
-        const bool okA = rowA < M, okB = rowB < M;
-        for (int t = 0; t < tiles_per_unit; ++t)
-            prune_tile<SUMS, true>(xa + t * 128, xb + t * 128, va + t * 64, vb + t * 64, slab + t * 512, okA,
-                                   okB, lut, numA, denA, numB, denB);
+    // The last tile's results stay in registers until after the row-sum hand-over below, so that
+    // the fence of that hand-over does not have to wait for the big value stores.
+    TileOut last;
+    uint16_t *va = nullptr, *vb = nullptr;
+    uint32_t* slab = nullptr;
+    const bool full_rows = row0 + PRUNE_ROWS <= M;
+    const bool okA = rowA < M, okB = rowB < M;
+    if (active) {
+        const int64_t kb0 = (int64_t)ks * tiles_per_unit;
+        // metadata slab of this row block inside block (row0/128, kb)
+        slab = reinterpret_cast<uint32_t*>(meta + ((row0 / 128) * kblocks + kb0) * 2048 +
+                                           ((row0 % 128) / 16) * 256 + lane * 4);
+        const uint16_t* xa = X + rowA * ldx + kb0 * 128 + q * 32;
+        const uint16_t* xb = xa + 8 * ldx;
+        va = values + rowA * (K / 2) + kb0 * 64 + q * 16;
+        vb = va + 8 * (K / 2);
+        for (int t = 0; t < tiles_per_unit; ++t) {
+            if (full_rows)
+                prune_tile_compute<SUMS, false>(xa, xb, true, true, lut, last, numA, denA, numB, denB);
+            else
+                prune_tile_compute<SUMS, true>(xa, xb, okA, okB, lut, last, numA, denA, numB, denB);
+            if (t + 1 < tiles_per_unit) {
+                prune_tile_store(last, va, vb, slab, okA, okB);
+                xa += 128; xb += 128; va += 64; vb += 64; slab += 512;
+            }
+        }
     }
 
     if constexpr (SUMS) {
@@ -215,51 +236,56 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
             numB += __shfl_xor_sync(0xffffffffu, numB, off);
             denB += __shfl_xor_sync(0xffffffffu, denB, off);
         }
-        if (q == 0) {
-            if (KS == 1) {
+        if (KS == 1) {
+            if (active) prune_tile_store(last, va, vb, slab, okA, okB);
+            if (active && q == 0) {
                 if (rowA < M) write_scale_or_sums(mode, rowA, numA, denA, row_scale, sums);
                 if (rowB < M) write_scale_or_sums(mode, rowB, numB, denB, row_scale, sums);
-            } else {
-                float* mine = partial + (rb16 * KS + ks) * 32;
-                *reinterpret_cast<float2*>(mine + 2 * r) = make_float2(numA, denA);
-                *reinterpret_cast<float2*>(mine + 2 * (r + 8)) = make_float2(numB, denB);
             }
+            return;
         }
-    } else {
-        if (row_scale != nullptr && ks == 0 && lane < 16 && row0 + lane < M) row_scale[row0 + lane] = 1.0f;
-    }
-}
-
-// One CTA per 16-row block: adds the KS partial sums of each row in a fixed order (16 strided
-// running sums per row, then those 16 in ascending order), so the result is reproducible.
-__global__ void __launch_bounds__(256)
-row_scale_kernel(const float* __restrict__ partial, int64_t M, int KS, int mode, float* __restrict__ row_scale,
-                 float* __restrict__ sums) {
-    __shared__ float2 red[16][16];
-    griddep_wait();  // launched early (programmatic dependent launch): partial sums must be complete
-    const int row = threadIdx.x & 15, jl = threadIdx.x >> 4;
-    const int64_t rb16 = blockIdx.x;
-    const float2* p = reinterpret_cast<const float2*>(partial) + rb16 * KS * 16 + row;
-    float num = 0.f, den = 0.f;
-    for (int j = jl; j < KS; j += 16) {
-        const float2 v = __ldcg(p + j * 16);
-        num += v.x;
-        den += v.y;
-    }
-    red[jl][row] = make_float2(num, den);
-    __syncthreads();
-    if (threadIdx.x < 16) {
-        const int64_t m = rb16 * 16 + threadIdx.x;
-        if (m < M) {
+        if (active && q == 0) {
+            float* mine = partial + (rb16 * KS + ks) * 32;
+            *reinterpret_cast<float2*>(mine + 2 * r) = make_float2(numA, denA);
+            *reinterpret_cast<float2*>(mine + 2 * (r + 8)) = make_float2(numB, denB);
+        }
+        // The last CTA of the row block to get here adds all partial sums, in a fixed order.  One
+        // thread fences and takes the ticket for the whole CTA (the barrier makes the other
+        // warps' stores its predecessors), so only its warp waits for the stores to drain.
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            const uint32_t t = atomicAdd(&tickets[rb16], 1u);
+            s_last = (t == (uint32_t)(ctas_per_rb - 1)) ? 1u : 0u;
+        }
+        __syncthreads();
+        if (active) prune_tile_store(last, va, vb, slab, okA, okB);
+        if (!s_last) return;
+        __threadfence();
+        const int row = tid & 15, jl = tid >> 4;  // 16 rows x (PRUNE_CTA_WARPS * 2) strided sums
+        const float2* pp = reinterpret_cast<const float2*>(partial) + rb16 * KS * 16 + row;
+        float num = 0.f, den = 0.f;
+        for (int j = jl; j < KS; j += PRUNE_CTA_WARPS * 2) {
+            const float2 v = __ldcg(pp + j * 16);
+            num += v.x;
+            den += v.y;
+        }
+        red[jl][row] = make_float2(num, den);
+        __syncthreads();
+        if (tid < 16 && row0 + tid < M) {
             num = 0.f;
             den = 0.f;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                num += red[j][threadIdx.x].x;
-                den += red[j][threadIdx.x].y;
+            for (int j = 0; j < PRUNE_CTA_WARPS * 2; ++j) {
+                num += red[j][tid].x;
+                den += red[j][tid].y;
             }
-            write_scale_or_sums(mode, m, num, den, row_scale, sums);
+            write_scale_or_sums(mode, row0 + tid, num, den, row_scale, sums);
         }
+        if (tid == 0) tickets[rb16] = 0;  // ready for the next launch
+    } else {
+        if (active) prune_tile_store(last, va, vb, slab, okA, okB);
+        if (row_scale != nullptr && ks == 0 && lane < 16 && row0 + lane < M) row_scale[row0 + lane] = 1.0f;
     }
 }
 
