@@ -120,8 +120,8 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
                       Cfg::BN_CTA, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_tmap_2d(&te, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, meta, rb * kblocks * 2, 256, 1024, 256, 2,
                       CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, 64,
-                      32, CU_TENSOR_MAP_SWIZZLE_128B))
+        !make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, Cfg::CH,
+                      32, Cfg::CH == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE))
         return LYNX_ERR_CUDA;
 
     GemmParams p;
@@ -193,13 +193,16 @@ lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int
                         cudaStream_t st) {
     int cfg = ctx->gemm_cfg;
     if (cfg == 0) {
-        // CTA-pair tiles 256 x {256, 192, 128}.  Pick the one with the smallest modelled time:
+        // CTA-pair tiles 256 x {256, 240, 192, 128}.  A sparse MMA takes the same time whatever its N
+        // (up to 256), so wide tiles win; 240 is the widest that still double-buffers the
+        // accumulator.  Pick the tile with the smallest modelled time:
         // rounds of tiles over the CTA pairs x (K blocks x measured time per K block + exposed
         // epilogue).  Per-K-block times (us) are measured B200 figures for each tile shape; the
         // 256-wide tile has one accumulator buffer, so its epilogue is not hidden.
         const int pairs = ctx->num_sms / 2;
         const double kb = (double)(K / 128);
-        struct { int id, bn; double t_kb, epi; } cand[3] = {{5, 256, 0.50, 3.0}, {4, 192, 0.415, 0.6}, {6, 128, 0.345, 0.5}};
+        struct { int id, bn; double t_kb, epi; } cand[4] = {
+            {7, 240, 0.465, 0.6}, {5, 256, 0.50, 3.0}, {4, 192, 0.415, 0.6}, {6, 128, 0.345, 0.5}};
         double best = 1e30;
         for (auto& c : cand) {
             const int64_t tiles = ((M + 255) / 256) * ((N + c.bn - 1) / c.bn);
@@ -216,6 +219,7 @@ lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int
         case 4: return launch_gemm_cfg<GemmCfg<192, 2, 4, 2>>(LYNX_GEMM_ARGS);
         case 5: return launch_gemm_cfg<GemmCfg<256, 2, 4, 1>>(LYNX_GEMM_ARGS);
         case 6: return launch_gemm_cfg<GemmCfg<128, 2, 5, 2>>(LYNX_GEMM_ARGS);
+        case 7: return launch_gemm_cfg<GemmCfg<240, 2, 4, 2>>(LYNX_GEMM_ARGS);
         default: return LYNX_ERR_INVALID_ARG;
     }
 #undef LYNX_GEMM_ARGS

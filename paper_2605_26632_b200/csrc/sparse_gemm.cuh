@@ -114,7 +114,11 @@ struct GemmCfg {
     static constexpr int B_BYTES = 2 * B_HALF_BYTES;
     static constexpr int E_BYTES = 2048;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
-    static constexpr int C_BOX_BYTES = 32 * 64 * 2;  // one warp's 32 x 64 bf16 store box
+    // epilogue chunk: 64 columns (128-byte swizzled staging rows) when BN allows, else 48 columns
+    // (96-byte unswizzled rows) -- BN = 240 is the widest tile that leaves room for two
+    // accumulator buffers plus the metadata columns in the 512 columns of tensor memory
+    static constexpr int CH = (BN % 64 == 0) ? 64 : 48;
+    static constexpr int C_BOX_BYTES = 32 * CH * 2;  // one warp's 32 x CH bf16 store box
     static constexpr int C_BYTES = 4 * CBUFS * C_BOX_BYTES;
     static constexpr int ACC_STAGES = (2 * BN + 4 * STAGES <= 512) ? 2 : 1;
     static constexpr int E_COL0 = ACC_STAGES * BN;  // metadata columns start after accumulators
@@ -122,8 +126,9 @@ struct GemmCfg {
     static constexpr int NUM_BARS = 2 * STAGES + 2 * ACC_STAGES;
     static constexpr int SMEM_BYTES = 1024 /*align slack*/ + STAGES * STAGE_BYTES + C_BYTES + 256;
     static constexpr int THREADS = 192;
-    static_assert(BN % (16 * CG) == 0 && BN <= 256, "tile N");
-    static_assert(BN % 64 == 0, "epilogue works on 64-column chunks");
+    static_assert(BN % 16 == 0 && (BN / CG) % 8 == 0 && BN <= 256, "tile N");
+    static_assert(BN % CH == 0, "epilogue works on whole chunks");
+    static_assert(C_BOX_BYTES % 1024 == 0, "staging boxes stay 1024-byte aligned");
     static_assert(B_HALF_BYTES % 1024 == 0, "swizzle atoms need 1024-byte aligned tiles");
     static_assert(E_COL0 % 4 == 0 && E_COL0 + 4 * STAGES <= TMEM_COLS, "tensor memory budget");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
@@ -309,7 +314,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
             // stream-K pieces: this thread's row of the pair tile inside an fp32 partial slot
             const size_t slot_floats = (size_t)Cfg::BM * CG * BN;
-            // layout of a slot: [64-column chunk][16-byte piece j][row of the pair tile] float4, so a
+            // layout of a slot: [CH-column chunk][16-byte piece j][row of the pair tile] float4, so a
             // warp's 32 rows of one piece are 512 contiguous bytes
             constexpr int SLOT_ROWS = Cfg::BM * CG;
             const size_t my_row_off = (size_t)((int)rank * Cfg::BM + q * 32 + lane);
@@ -325,13 +330,17 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 if (!alive) break;
             }
 #pragma unroll 1
-            for (int c = 0; c < BN / 64; ++c) {
-                const int n0 = tn * BN + c * 64;
-                uint32_t v[64];
-                tmem_ld_32x32b_x32(t_row + c * 64, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-                tmem_ld_32x32b_x32(t_row + c * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+            constexpr int CH = Cfg::CH;
+            for (int c = 0; c < BN / CH; ++c) {
+                const int n0 = tn * BN + c * CH;
+                uint32_t v[CH];
+                tmem_ld_32x32b_x32(t_row + c * CH, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                if constexpr (CH == 64)
+                    tmem_ld_32x32b_x32(t_row + c * CH + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+                else
+                    tmem_ld_32x32b_x16(t_row + c * CH + 32, *reinterpret_cast<uint32_t(*)[16]>(&v[32]));
                 tmem_ld_wait();
-                if (c == BN / 64 - 1) {
+                if (c == BN / CH - 1) {
                     // accumulator fully read: hand it back to the MMA issuer
                     tc_fence_before();
                     __syncwarp();
@@ -343,9 +352,9 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 if (w.kind == 1) {
                     // partial piece: raw fp32 accumulators to this cluster's slot
                     float4* dst = reinterpret_cast<float4*>(p.sk_partial + (size_t)cluster_id * slot_floats) +
-                                  (size_t)c * 16 * SLOT_ROWS + my_row_off;
+                                  (size_t)c * (CH / 4) * SLOT_ROWS + my_row_off;
 #pragma unroll
-                    for (int j = 0; j < 16; ++j)
+                    for (int j = 0; j < CH / 4; ++j)
                         __stcg(dst + (size_t)j * SLOT_ROWS, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
                                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
                     continue;
@@ -355,12 +364,12 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     for (int cc = w.first_contrib; cc < cluster_id; ++cc) {
                         if (!sched.has_tail(cc)) continue;
                         const float4* src = reinterpret_cast<const float4*>(p.sk_partial + (size_t)cc * slot_floats) +
-                                            (size_t)c * 16 * SLOT_ROWS + my_row_off;
-                        float4 pa[16];
+                                            (size_t)c * (CH / 4) * SLOT_ROWS + my_row_off;
+                        float4 pa[CH / 4];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) pa[j] = __ldcg(src + (size_t)j * SLOT_ROWS);
+                        for (int j = 0; j < CH / 4; ++j) pa[j] = __ldcg(src + (size_t)j * SLOT_ROWS);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
+                        for (int j = 0; j < CH / 4; ++j) {
                             const float4 a = pa[j];
                             v[4 * j] = __float_as_uint(__uint_as_float(v[4 * j]) + a.x);
                             v[4 * j + 1] = __float_as_uint(__uint_as_float(v[4 * j + 1]) + a.y);
@@ -375,7 +384,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 __syncwarp();
                 const uint32_t cbuf = cbuf0 + cb * Cfg::C_BOX_BYTES;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {  // 8 columns (16 bytes of output) at a time
+                for (int j = 0; j < CH / 8; ++j) {  // 8 columns (16 bytes of output) at a time
                     const int n = n0 + j * 8;
                     float b[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                     float r[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -402,8 +411,10 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                         const float y1 = fmaf(s, __uint_as_float(v[j * 8 + 2 * e + 1]), b[2 * e + 1]) + r[2 * e + 1];
                         o[e] = pack_bf16x2(y0, y1);
                     }
-                    // 128-byte rows, 16-byte chunk index XOR (row % 8): the 128-byte swizzle
-                    sts128(cbuf + lane * 128 + ((j ^ (lane & 7)) << 4), o[0], o[1], o[2], o[3]);
+                    if constexpr (CH == 64)  // 128-byte rows, 16-byte chunk index XOR (row % 8): the 128-byte swizzle
+                        sts128(cbuf + lane * 128 + ((j ^ (lane & 7)) << 4), o[0], o[1], o[2], o[3]);
+                    else  // dense 96-byte rows for the unswizzled 48-column box
+                        sts128(cbuf + lane * (CH * 2) + (j << 4), o[0], o[1], o[2], o[3]);
                 }
                 fence_proxy_async_smem();
                 __syncwarp();

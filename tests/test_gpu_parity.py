@@ -164,9 +164,9 @@ def test_tiny_config_full_oracle(lx, mode, with_bias, with_res):
     assert torch.equal(Y, Y2)
 
 
-@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6, 7])
 def test_every_tile_configuration(cfg, monkeypatch):
-    """All compiled tile shapes (one- and two-CTA MMAs, 128/192/256 columns) give the same answer."""
+    """All compiled tile shapes (one- and two-CTA MMAs, 128/192/240/256 columns) give the same answer."""
     from paper_2605_26632_b200 import binding
 
     monkeypatch.setenv("LYNX_GEMM_CFG", str(cfg))
@@ -184,7 +184,7 @@ def test_every_tile_configuration(cfg, monkeypatch):
         ctx.close()
 
 
-@pytest.mark.parametrize("cfg", [4, 5])
+@pytest.mark.parametrize("cfg", [4, 5, 7])
 def test_stream_k_tail_matches_oracle_and_is_deterministic(cfg, monkeypatch):
     """Optional stream-K tail (leftover tiles split along K, fp32 partial tiles added in fixed
     order): same answer within tolerance, bit-identical run to run."""
