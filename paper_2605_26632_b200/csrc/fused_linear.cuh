@@ -160,6 +160,7 @@ fused_linear_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
+            if (!ok) bounded_delay_ns(200000);  // let the copies in flight land before teardown
         }
     } else if (warp >= 6) {
         // ------------------------------------------------------------------ pruners -----------

@@ -114,6 +114,13 @@ __device__ __forceinline__ bool flag_wait(const uint32_t* flag, uint32_t want, v
     }
 }
 
+// After a timeout the producer gives its bulk copies still in flight a bounded time to land
+// before the CTA tears down (they complete on their own; nothing else can be done about them).
+__device__ __forceinline__ void bounded_delay_ns(uint64_t ns) {
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < ns) __nanosleep(256);
+}
+
 // ---------------------------------------------------------------------------- TMA ------------
 
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {

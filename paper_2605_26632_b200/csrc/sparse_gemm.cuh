@@ -244,7 +244,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
-            (void)issued;
+            if (!ok && issued) bounded_delay_ns(200000);  // let the copies in flight land before teardown
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer --------

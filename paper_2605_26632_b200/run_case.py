@@ -1,6 +1,6 @@
 """Runs a few launches of one kernel of the path on a named synthetic workload.
 
-    python -m paper_2605_26632_b200.run_case --kernel prune|gemm|layer --workload mlp_down [--iters 3]
+    python -m paper_2605_26632_b200.run_case --kernel prune|gemm|layer|fused --workload mlp_down [--iters 3]
 
 Meant as the small, self-terminating command to put under a profiler (one kernel, a few launches,
 well under a GB on the device), and as a minimal usage example of the binding.
@@ -16,7 +16,7 @@ from . import binding, inputs
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="layer", choices=["prune", "gemm", "layer"])
+    ap.add_argument("--kernel", default="layer", choices=["prune", "gemm", "layer", "fused"])
     ap.add_argument("--workload", default="mlp_down")
     ap.add_argument("--M", type=int, default=0, help="override the number of token rows")
     ap.add_argument("--iters", type=int, default=3)
@@ -38,6 +38,8 @@ def main():
             lx.prune_compress(X, args.comp, values, meta, scale)
         if args.kernel in ("gemm", "layer"):
             lx.sparse_linear(values, meta, W, b, scale, None, Y)
+        if args.kernel == "fused":
+            lx.act_sparse_linear(X, W, b, args.comp, None, Y, binding.FUSE_FUSED)
     torch.cuda.synchronize()
     assert lx.last_error() == 0
     print(f"ran {args.iters} x {args.kernel} on {args.workload} (M={M}, K={wl.K}, N={wl.N}); "
