@@ -305,7 +305,7 @@ def main():
     prune_ms = [evs[i][0].elapsed_time(evs[i][1]) for i in probed]
     gemm_ms = [evs[i][1].elapsed_time(evs[i][2]) for i in probed]
 
-    # prune/compress (+ its finalize launch) alone, back to back over the rotating sets: the
+    # prune/compress (row scale finalized in the same launch) alone, back to back over the rotating sets: the
     # per-launch time that the HBM roofline of that kernel is judged on
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for i in range(3):
@@ -396,7 +396,7 @@ def main():
         "roofline_prune": {"bound": "hbm", "kernel": "prune_compress_kernel", "achieved": prune_gbs,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": prune_gbs / peaks["hbm_gbs"],
                            "frac_of_8TBs_nominal": prune_gbs / 8000.0, "bytes_per_launch": prune_bytes, "ms_per_launch": prune_loop_ms,
-                           "how": "back-to-back loop of lynx_prune_compress (prune + row-scale finalize kernels) over "
+                           "how": "back-to-back loop of lynx_prune_compress (one launch: select, compress, row sums, scale) over "
                                   "rotating buffers, CUDA events; the in-step figure is kernels.prune_compress_ms",
                            "peak_kind": f"hbm_gbs ({peaks['source']})"},
         "clocks": clocks,

@@ -113,7 +113,13 @@ LYNX_API lynx_status lynx_reserve(lynx_ctx* ctx, int64_t M, int64_t N, int64_t K
  *         row-major form for inspection.
  *   row_scale (may be NULL when mode == LYNX_COMP_NONE): [M] fp32, s_m per `mode`
  *         (ROW: per row; TENSOR: the same global s in every entry; NONE: 1.0 if non-NULL).
- * TENSOR mode uses the context's scratch (2 floats per row).
+ * Alignment for this step: X and values 32-byte aligned, ldx % 16 == 0 (32-byte vector
+ * accesses), meta 16-byte aligned; violations return LYNX_ERR_ALIGNMENT.
+ * ROW and TENSOR modes use the context's scratch: partial sums of each 16-row block per run of
+ * K blocks, one ticket word per 16-row block (the last CTA of a block adds the partial sums in
+ * ascending K order, so row_scale is reproducible bit for bit, and resets the ticket), and in
+ * TENSOR mode 2 floats per row.  The scratch is grown on demand (see lynx_reserve).
+ * With the ticket area fixed at 1 MB, M > 4194304 returns LYNX_ERR_UNSUPPORTED_SHAPE.
  */
 LYNX_API lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
                                          int64_t ldx, void* values, void* meta, float* row_scale,
@@ -130,12 +136,15 @@ LYNX_API lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M
  *   - Works on the CURRENT device.  The first call on each device looks up the array's device
  *     address (cudaGetSymbolAddress) and caches it; make that first call before any stream
  *     capture begins.
- *   - Shapes whose scratch need -- ceil(M/128)*8 * (K/128)/t * 128 bytes of partial sums, t the
- *     K blocks per warp the library picks, plus 8*M bytes in LYNX_COMP_TENSOR mode -- exceeds
+ *   - Shapes whose scratch need -- a fixed 64 KB ticket area (one word per 16 rows, so
+ *     M <= 262144), plus ceil(M/128)*8 * (K/128)/t * 128 bytes of partial sums, t the K blocks
+ *     per warp the library picks, plus 8*M bytes in LYNX_COMP_TENSOR mode -- exceeds
  *     LYNX_STATIC_SCRATCH_BYTES are refused with LYNX_ERR_WORKSPACE; LYNX_COMP_NONE needs none.
- *   - Every call shares the one array and finds the previous call's contents in it; nothing in
- *     it has to start at zero (each call overwrites what it later reads).  Two calls that overlap
- *     on the GPU (different streams, no ordering between them) race on it: order them.
+ *   - Every call shares the one array and finds the previous call's contents in it.  The sums
+ *     are overwritten before they are read; the ticket words start at zero (the array is
+ *     zero-initialised when the library is loaded) and every launch leaves them at zero.  Two
+ *     calls that overlap on the GPU (different streams, no ordering between them) race on it:
+ *     order them.
  *   - No device-side error word: the kernels involved have no waits that can time out.
  * Arguments, layouts, alignment rules and results are exactly those of lynx_prune_compress. */
 #define LYNX_STATIC_SCRATCH_BYTES (8u << 20)
