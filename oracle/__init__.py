@@ -208,17 +208,30 @@ def epilogue(acc, M, s=None, bias=None, Yr=None, rows=None) -> np.ndarray:
     return Y
 
 
-def lora_residual(X, LB, LA) -> np.ndarray:
+def lora_residual(X, LB, LA, rows=None) -> np.ndarray:
+    """Y_r = (X L_B^T) L_A^T in fp32 for `rows` (None = all rows)."""
     X, M, K = _check_x(X)
     LB = _u16(LB, "LB")
     LA = _u16(LA, "LA")
     R = LB.shape[0]
     N = LA.shape[0]
     assert LB.shape == (R, K) and LA.shape == (N, R) and R <= 512
-    Yr = np.empty((M, N), dtype=np.float32)
-    _load().oracle_lora_residual(_p(X), _i64(M), _i64(K), _i64(K), _p(LB), _i64(R), _p(LA), _i64(N),
-                                 _p(Yr))
+    r, nr = _rows(rows, M)
+    Yr = np.empty((nr, N), dtype=np.float32)
+    _load().oracle_lora_residual_rows(_p(X), _i64(M), _i64(K), _i64(K), _p(LB), _i64(R), _p(LA), _i64(N),
+                                      _p(r), _i64(nr), _p(Yr))
     return Yr
+
+
+def act_sparse_linear_lora(X, W, LA, LB, bias=None, comp_mode=COMP_NONE, Yr=None, rows=None):
+    """Whole path of Algorithm 1 with the LoRA branch: Y = s * (X~ W^T) + b [+ Yr] + X (L_A L_B)^T."""
+    out = act_sparse_linear(X, W, bias=bias, comp_mode=comp_mode, Yr=Yr, rows=rows)
+    lora = lora_residual(X, LB, LA, rows=rows)
+    Y = np.ascontiguousarray(out["Y"], dtype=np.float32)
+    _load().oracle_add_lora(_p(Y), _p(lora), _i64(Y.shape[0]), _i64(Y.shape[1]))
+    out["Y"] = Y
+    out["lora"] = lora
+    return out
 
 
 def act_sparse_linear(X, W, bias=None, comp_mode=COMP_NONE, Yr=None, rows=None):

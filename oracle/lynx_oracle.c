@@ -287,13 +287,17 @@ ORACLE_API void oracle_epilogue(const float* acc, int64_t N, const int64_t* rows
     }
 }
 
-/* ---- Step 7 (optional addend producer): LoRA residual on the DENSE X ------------------
- * Yr = (X L_B^T) L_A^T, L_B is R x K, L_A is N x R, all bf16, fp32 accumulation.        */
-ORACLE_API void oracle_lora_residual(const uint16_t* X, int64_t M, int64_t K, int64_t ldx,
-                                     const uint16_t* LB, int64_t R, const uint16_t* LA, int64_t N,
-                                     float* Yr) {
+/* ---- Step 7: LoRA residual on the DENSE X (Algorithm 1 lines 5-6: Y_r = X (L_A L_B)^T) ----
+ * Yr = (X L_B^T) L_A^T, L_B is R x K, L_A is N x R, all bf16, fp32 accumulation, nothing
+ * rounded in between.  Computed for the rows listed in `rows` (NULL = all M rows, in order);
+ * Yr is n_rows x N.                                                                        */
+ORACLE_API void oracle_lora_residual_rows(const uint16_t* X, int64_t M, int64_t K, int64_t ldx,
+                                          const uint16_t* LB, int64_t R, const uint16_t* LA, int64_t N,
+                                          const int64_t* rows, int64_t n_rows, float* Yr) {
+    if (!rows) n_rows = M;
 #pragma omp parallel for schedule(dynamic, 1)
-    for (int64_t m = 0; m < M; ++m) {
+    for (int64_t i = 0; i < n_rows; ++i) {
+        const int64_t m = rows ? rows[i] : i;
         float t[512];
         for (int64_t r = 0; r < R && r < 512; ++r) {
             float a = 0.0f;
@@ -304,9 +308,21 @@ ORACLE_API void oracle_lora_residual(const uint16_t* X, int64_t M, int64_t K, in
         for (int64_t n = 0; n < N; ++n) {
             float a = 0.0f;
             for (int64_t r = 0; r < R && r < 512; ++r) a += t[r] * bf16_to_f32(LA[n * R + r]);
-            Yr[m * N + n] = a;
+            Yr[i * N + n] = a;
         }
     }
+}
+
+ORACLE_API void oracle_lora_residual(const uint16_t* X, int64_t M, int64_t K, int64_t ldx,
+                                     const uint16_t* LB, int64_t R, const uint16_t* LA, int64_t N,
+                                     float* Yr) {
+    oracle_lora_residual_rows(X, M, K, ldx, LB, R, LA, N, NULL, M, Yr);
+}
+
+/* ---- Algorithm 1 line 6 with the LoRA branch kept in fp32: Y += Y_r -----------------------
+ * Y and lora are n_rows x N; the sum is one fp32 addition per element.                     */
+ORACLE_API void oracle_add_lora(float* Y, const float* lora, int64_t n_rows, int64_t N) {
+    for (int64_t i = 0; i < n_rows * N; ++i) Y[i] = Y[i] + lora[i];
 }
 
 /* ---- Whole path for a set of rows: steps 1, 2, 4, 5, 6 in that order -------------------

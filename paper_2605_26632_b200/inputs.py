@@ -42,10 +42,15 @@ WORKLOADS = {
 
 SWEEP_M = (1024, 4096, 8192, 16384)
 SWEEP_KN = ((3072, 9216), (3072, 3072), (3072, 12288), (12288, 3072))
+# Linear shapes that only the other two DiT families have: FLUX.1-dev single-stream blocks
+# ((3072, 21504) fused QKV+MLP-up, (15360, 3072) fused Out+MLP-down) and Z-Image (hidden 3840,
+# MLP 10240: N = 10240 is not a multiple of any tile width, so it exercises the column tail).
+OTHER_FAMILY_KN = ((3072, 21504), (15360, 3072), (3840, 3840), (3840, 10240), (10240, 3840))
+OTHER_FAMILY_M = 4096
 
 
 def sweep_workload(M: int, K: int, N: int, index: int = 0) -> Workload:
-    dist = "gelu_chan" if K == 12288 else "outlier"
+    dist = "gelu_chan" if K >= 10240 else "outlier"
     return Workload(f"sweep_M{M}_K{K}_N{N}", M, K, N, dist, 5000 + index)
 
 

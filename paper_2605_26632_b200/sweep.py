@@ -40,6 +40,7 @@ def main():
     Ms = (4096,) if args.quick else inputs.SWEEP_M
     shapes = [(M, K, N) for M in Ms for (K, N) in inputs.SWEEP_KN]
     shapes += [(4352, 3072, 9216), (4352, 3072, 3072)]
+    shapes += [(inputs.OTHER_FAMILY_M, K, N) for (K, N) in inputs.OTHER_FAMILY_KN]
     if not args.quick:
         shapes += [(M, K, M) for M in (2048, 4096, 8192) for K in (3072, 12288)]  # the paper's kernel grid
     print("| M | K | N | prune us | prune GB/s | GEMM us | GEMM TF | layer us | layer TF | fused us | fused TF | "

@@ -370,6 +370,13 @@ def test_token_sweep(lx, M, K, N):
     _full_size_case(lx, inputs.sweep_workload(M, K, N, idx), 16)
 
 
+@pytest.mark.parametrize("K,N", inputs.OTHER_FAMILY_KN)
+def test_other_dit_family_shapes(lx, K, N):
+    """FLUX.1-dev single-stream and Z-Image linear shapes (full size, sampled rows)."""
+    idx = 100 + inputs.OTHER_FAMILY_KN.index((K, N))
+    _full_size_case(lx, inputs.sweep_workload(inputs.OTHER_FAMILY_M, K, N, idx), 16)
+
+
 # ------------------------------------------------------------------ host-side error reporting ---
 
 def test_argument_errors_are_reported_not_launched(lx):

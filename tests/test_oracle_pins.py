@@ -326,6 +326,59 @@ def test_lora_residual_matches_library_matmul():
     np.testing.assert_allclose(got, ref.numpy(), rtol=1e-5, atol=1e-6)
 
 
+def test_lora_rows_subset_equals_full_rows():
+    g = torch.Generator().manual_seed(12)
+    M, K, R, N = 20, 128, 8, 24
+    x = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    lb = (torch.randn(R, K, generator=g) * 0.1).to(torch.bfloat16)
+    la = (torch.randn(N, R, generator=g) * 0.1).to(torch.bfloat16)
+    full = oracle.lora_residual(inputs.as_u16(x), inputs.as_u16(lb), inputs.as_u16(la))
+    rows = np.array([19, 0, 7], dtype=np.int64)
+    sub = oracle.lora_residual(inputs.as_u16(x), inputs.as_u16(lb), inputs.as_u16(la), rows=rows)
+    assert (sub == full[rows]).all()
+
+
+def test_lora_path_uses_the_dense_x_not_the_pruned_one():
+    """W = 0 leaves only the LoRA branch: Y must be the DENSE product X (L_A L_B)^T (Algorithm 1
+    line 5 applies the low-rank term to X, not to S(X)); a branch fed with the pruned X fails."""
+    g = torch.Generator().manual_seed(13)
+    M, K, R, N = 16, 128, 8, 40
+    x = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    w = torch.zeros(N, K, dtype=torch.bfloat16)
+    lb = (torch.randn(R, K, generator=g) * 0.2).to(torch.bfloat16)
+    la = (torch.randn(N, R, generator=g) * 0.2).to(torch.bfloat16)
+    out = oracle.act_sparse_linear_lora(inputs.as_u16(x), inputs.as_u16(w), inputs.as_u16(la), inputs.as_u16(lb),
+                                        comp_mode=oracle.COMP_ROW)
+    dense = (x.double() @ lb.double().T) @ la.double().T
+    np.testing.assert_allclose(out["Y"], dense.numpy(), rtol=2e-5, atol=2e-6)
+    mask = torch.from_numpy(oracle.topk24_mask(inputs.as_u16(x)).astype(np.float64))
+    pruned = ((x.double() * mask) @ lb.double().T) @ la.double().T
+    assert np.abs(out["Y"] - pruned.numpy()).max() > 1e-2
+
+
+def test_lora_path_on_sparse_input_is_a_dense_linear_with_merged_weights():
+    """On an input that already is 2:4 sparse the layer is exact (s = 1, mask = support), so
+    Y = X (W + L_A L_B)^T + b: the LoRA term is neither scaled by s nor dropped, and it is
+    added once."""
+    g = torch.Generator().manual_seed(14)
+    M, K, R, N = 12, 256, 16, 24
+    x = torch.randn(M, K, generator=g)
+    keep = torch.zeros(M, K // 4, 4)
+    keep[..., 0] = 1
+    keep[..., 2] = 1
+    x = torch.where(keep.reshape(M, K) > 0, x, torch.zeros(())).to(torch.bfloat16)
+    w = (torch.randn(N, K, generator=g) * K ** -0.5).to(torch.bfloat16)
+    b = (torch.randn(N, generator=g) * 0.1).to(torch.bfloat16)
+    lb = (torch.randn(R, K, generator=g) * 0.1).to(torch.bfloat16)
+    la = (torch.randn(N, R, generator=g) * 0.1).to(torch.bfloat16)
+    for mode in (oracle.COMP_NONE, oracle.COMP_ROW, oracle.COMP_TENSOR):
+        out = oracle.act_sparse_linear_lora(inputs.as_u16(x), inputs.as_u16(w), inputs.as_u16(la), inputs.as_u16(lb),
+                                            bias=inputs.as_u16(b), comp_mode=mode)
+        merged = w.double() + la.double() @ lb.double()
+        ref = x.double() @ merged.T + b.double()
+        np.testing.assert_allclose(out["Y"], ref.numpy(), rtol=1e-4, atol=1e-5)
+
+
 def test_bf16_rounding_routine_matches_torch():
     g = torch.Generator().manual_seed(3)
     v = torch.randn(4096, generator=g) * 10
