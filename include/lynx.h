@@ -185,6 +185,45 @@ LYNX_API lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_ho
                                                  const void* bias, lynx_comp_mode mode, void* Y_host,
                                                  lynx_fuse_mode fuse, void* stream);
 
+/* ---- low-rank branch (Algorithm 1 lines 5-6: Y = Y_s + Y_r, Y_r = X (L_A L_B)^T; the
+ *      interleaved-LoRA kernel optimisation of the kernel section) -------------------------------
+ * L_B is R x K bf16 row-major (leading dimension ldlb), L_A is N x R bf16 row-major (ldla);
+ * R is 64 or 128 (others: LYNX_ERR_UNSUPPORTED_SHAPE).  The branch reads the DENSE X.  Y_r is
+ * never written to memory: the down projection T = X L_B^T is computed once per layer and the
+ * up projection T L_A^T is added inside the sparse GEMM's accumulator by dense tensor-core
+ * steps, so that
+ *   Y[m, n] = bf16_rne( s_m * sum_k X~[m,k] W[n,k] + sum_r T[m,r] L_A[n,r] + bias[n] + Y_r'[m,n] )
+ * (Y_r' = the optional comp->residual addend).  Because the epilogue multiplies the whole
+ * accumulator by s_m, T is stored pre-divided:
+ *
+ * lynx_lora_down:  T[m, r] = bf16_rne( (sum_k X[m,k] L_B[r,k]) / s_m ), fp32 accumulation on the
+ *   dense tensor cores; row_scale == NULL means s_m = 1; s_m == 0 gives T = 0.  T is M x R bf16,
+ *   leading dimension ldt (>= R, multiple of 8), owned by the caller.  Uses the context's
+ *   low-rank workspace (fp32 partials of the K splits; grown on demand, see lynx_reserve_lora)
+ *   and a ticket word per 128-row block (M <= 2097152).  The result does not depend on the
+ *   order in which CTAs finish.
+ * lynx_sparse_linear_lora:  lynx_sparse_linear plus the T L_A^T term; T must come from
+ *   lynx_lora_down called with the same row_scale that comp carries.
+ * lynx_act_sparse_linear_lora:  the whole layer: prune/compress, down projection, sparse GEMM
+ *   with the low-rank steps, back to back on `stream`, intermediates in the context's scratch.
+ * Pointers and leading dimensions follow the 16-byte rule of the other entry points.
+ */
+LYNX_API lynx_status lynx_reserve_lora(lynx_ctx* ctx, int64_t M, int64_t K, int64_t R);
+LYNX_API lynx_status lynx_lora_down(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx,
+                                    const void* LB, int64_t R, int64_t ldlb, const float* row_scale,
+                                    void* T, int64_t ldt, void* stream);
+LYNX_API lynx_status lynx_sparse_linear_lora(lynx_ctx* ctx, const void* values, const void* meta,
+                                             int64_t M, int64_t K, const void* W, int64_t N,
+                                             int64_t ldw, const void* bias, const lynx_comp* comp,
+                                             const void* T, int64_t ldt, const void* LA, int64_t R,
+                                             int64_t ldla, void* Y, int64_t ldy, void* stream);
+LYNX_API lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
+                                                 int64_t ldx, const void* W, int64_t N, int64_t ldw,
+                                                 const void* bias, const void* LA, int64_t ldla,
+                                                 const void* LB, int64_t ldlb, int64_t R,
+                                                 lynx_comp_mode mode, const void* residual,
+                                                 int64_t ldr, void* Y, int64_t ldy, void* stream);
+
 /* ---- inspection helpers ------------------------------------------------------------------------ */
 
 /* Hardware-order metadata -> canonical form: uint16 [M x K/16], nibble (g%4) of group g in bits

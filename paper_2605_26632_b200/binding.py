@@ -22,6 +22,7 @@ EXPORTS = [
     "lynx_meta_bytes", "lynx_workspace_bytes", "lynx_reserve", "lynx_prune_compress",
     "lynx_sparse_linear", "lynx_act_sparse_linear", "lynx_act_sparse_linear_host",
     "lynx_meta_to_canonical", "lynx_decompress", "lynx_launch_count", "lynx_prune_compress_static",
+    "lynx_reserve_lora", "lynx_lora_down", "lynx_sparse_linear_lora", "lynx_act_sparse_linear_lora",
 ]
 
 
@@ -72,6 +73,12 @@ def load_library() -> ctypes.CDLL:
     lib.lynx_meta_to_canonical.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.lynx_decompress.argtypes = [vp, vp, vp, i64, i64, vp, vp]
     lib.lynx_prune_compress_static.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
+    lib.lynx_reserve_lora.argtypes = [vp, i64, i64, i64]
+    lib.lynx_lora_down.argtypes = [vp, vp, i64, i64, i64, vp, i64, i64, vp, vp, i64, vp]
+    lib.lynx_sparse_linear_lora.argtypes = [vp, vp, vp, i64, i64, vp, i64, i64, vp, ctypes.POINTER(_Comp), vp,
+                                            i64, vp, i64, i64, vp, i64, vp]
+    lib.lynx_act_sparse_linear_lora.argtypes = [vp, vp, i64, i64, i64, vp, i64, i64, vp, vp, i64, vp, i64, i64,
+                                                i32, vp, i64, vp, i64, vp]
     lib.lynx_launch_count.argtypes = [vp]
     lib.lynx_launch_count.restype = i64
     _lib = lib
@@ -223,6 +230,60 @@ class Lynx:
                                                      _ptr(bias), mode, _ptr(Y_host), fuse, _stream()),
                "lynx_act_sparse_linear_host")
         return Y_host
+
+    # -- low-rank branch -----------------------------------------------------------------------
+    def reserve_lora(self, M: int, K: int, R: int):
+        _check(self._lib.lynx_reserve_lora(self._h, M, K, R), "lynx_reserve_lora")
+
+    def lora_down(self, X: torch.Tensor, LB: torch.Tensor, row_scale=None, out=None) -> torch.Tensor:
+        """T = bf16((X L_B^T) / s): [M, R]."""
+        _bf16_2d(X, "X")
+        _bf16_2d(LB, "LB")
+        M, K = X.shape
+        R = LB.shape[0]
+        if out is None:
+            out = torch.empty((M, R), dtype=torch.bfloat16, device=X.device)
+        _check(self._lib.lynx_lora_down(self._h, _ptr(X), M, K, X.stride(0), _ptr(LB), R, LB.stride(0),
+                                        _ptr(row_scale), _ptr(out), out.stride(0), _stream()), "lynx_lora_down")
+        return out
+
+    def sparse_linear_lora(self, values: torch.Tensor, meta: torch.Tensor, W: torch.Tensor, T: torch.Tensor,
+                           LA: torch.Tensor, bias=None, row_scale=None, residual=None, out=None) -> torch.Tensor:
+        _bf16_2d(values, "values")
+        _bf16_2d(W, "W")
+        _bf16_2d(T, "T")
+        _bf16_2d(LA, "LA")
+        M, K = values.shape[0], values.shape[1] * 2
+        N = W.shape[0]
+        R = LA.shape[1]
+        if out is None:
+            out = torch.empty((M, N), dtype=torch.bfloat16, device=values.device)
+        comp = _Comp(None if row_scale is None else row_scale.data_ptr(),
+                     None if residual is None else residual.data_ptr(),
+                     0 if residual is None else residual.stride(0))
+        _check(self._lib.lynx_sparse_linear_lora(self._h, _ptr(values), _ptr(meta), M, K, _ptr(W), N, W.stride(0),
+                                                 _ptr(bias), ctypes.byref(comp), _ptr(T), T.stride(0), _ptr(LA), R,
+                                                 LA.stride(0), _ptr(out), out.stride(0), _stream()),
+               "lynx_sparse_linear_lora")
+        return out
+
+    def act_sparse_linear_lora(self, X: torch.Tensor, W: torch.Tensor, LA: torch.Tensor, LB: torch.Tensor,
+                               bias=None, mode: int = COMP_NONE, residual=None, out=None) -> torch.Tensor:
+        _bf16_2d(X, "X")
+        _bf16_2d(W, "W")
+        _bf16_2d(LA, "LA")
+        _bf16_2d(LB, "LB")
+        M, K = X.shape
+        N = W.shape[0]
+        R = LB.shape[0]
+        if out is None:
+            out = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+        _check(self._lib.lynx_act_sparse_linear_lora(self._h, _ptr(X), M, K, X.stride(0), _ptr(W), N, W.stride(0),
+                                                     _ptr(bias), _ptr(LA), LA.stride(0), _ptr(LB), LB.stride(0), R,
+                                                     mode, _ptr(residual),
+                                                     0 if residual is None else residual.stride(0), _ptr(out),
+                                                     out.stride(0), _stream()), "lynx_act_sparse_linear_lora")
+        return out
 
     # -- inspection ----------------------------------------------------------------------------
     def meta_to_canonical(self, meta: torch.Tensor, M: int, K: int) -> torch.Tensor:

@@ -13,6 +13,7 @@
 #include "prune_compress.cuh"
 #include "sparse_gemm.cuh"
 #include "fused_linear.cuh"
+#include "lora_down.cuh"
 
 using namespace lynx;
 
@@ -24,6 +25,8 @@ struct lynx_ctx {
     void* scratch = nullptr;  // compressed operands, scale, sums, host staging mirrors
     size_t scratch_bytes = 0;
     uint32_t* tickets = nullptr;  // one word per 16-row block (prune finalize), zero between launches
+    void* lora_ws = nullptr;      // low-rank branch: [fp32 partials of the down projection][T]
+    size_t lora_ws_bytes = 0;
     float* sk_partial = nullptr;  // stream-K partial tiles (one slot per cluster) + ready words
     uint32_t* sk_flags = nullptr;
     uint32_t sk_epoch = 0;
@@ -82,6 +85,16 @@ lynx_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? LYNX_OK : LYNX_ER
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 constexpr size_t PRUNE_TICKET_BYTES = 1u << 20;  // 262144 row blocks of 16 rows = 4M rows
+constexpr size_t LORA_TICKET_BYTES = 64u << 10;  // after the prune tickets: 16384 row blocks of 128 rows
+
+// Low-rank branch operands of the GEMM: T = (X L_B^T) / s [M x R] bf16 and L_A [N x R] bf16.
+struct LoraArgs {
+    const void* T;
+    int64_t ldt;
+    const void* LA;
+    int64_t ldla;
+    int R;
+};
 
 // Scratch layout for (M, N, K):
 // [partial row sums][sums 2M floats][values][meta][row_scale M floats][X stage][Y stage]
@@ -111,8 +124,8 @@ ScratchLayout scratch_layout(int64_t M, int64_t N, int64_t K) {
 template <class Cfg>
 lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
                             const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
-                            void* Y, int64_t ldy, cudaStream_t st) {
-    CUtensorMap ta, tb, te, ty;
+                            const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st) {
+    CUtensorMap ta, tb, te, ty, tt, tla;
     const uint64_t rb = (uint64_t)((M + 127) / 128), kblocks = (uint64_t)(K / 128);
     if (!make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, values, (uint64_t)M, (uint64_t)(K / 2),
                       (uint64_t)K, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
@@ -123,8 +136,19 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
         !make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, Cfg::CH,
                       32, Cfg::CH == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE))
         return LYNX_ERR_CUDA;
+    if (lora) {
+        if (!make_tmap_2d(&tt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->T, (uint64_t)M, (uint64_t)lora->R,
+                          (uint64_t)lora->ldt * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap_2d(&tla, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->LA, (uint64_t)N, (uint64_t)lora->R,
+                          (uint64_t)lora->ldla * 2, 64, Cfg::BN_CTA, CU_TENSOR_MAP_SWIZZLE_128B))
+            return LYNX_ERR_CUDA;
+    } else {
+        tt = ta;  // never read: lora_steps = 0
+        tla = tb;
+    }
 
     GemmParams p;
+    p.lora_steps = lora ? lora->R / 64 : 0;
     p.M = M; p.N = N; p.K = K;
     p.row_scale = comp ? comp->row_scale : nullptr;
     p.bias = static_cast<const uint16_t*>(bias);
@@ -182,15 +206,15 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     attr[1].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, te, ty, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, te, ty, tt, tla, p);
     if (e != cudaSuccess) return LYNX_ERR_CUDA;
     ctx->launches++;
     return LYNX_OK;
 }
 
 lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K, const void* W,
-                        int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp, void* Y, int64_t ldy,
-                        cudaStream_t st) {
+                        int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp, const LoraArgs* lora, void* Y,
+                        int64_t ldy, cudaStream_t st) {
     int cfg = ctx->gemm_cfg;
     if (cfg == 0) {
         // CTA-pair tiles 256 x {256, 240, 192, 128}.  A sparse MMA takes the same time whatever its N
@@ -207,11 +231,11 @@ lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int
         for (auto& c : cand) {
             const int64_t tiles = ((M + 255) / 256) * ((N + c.bn - 1) / c.bn);
             const double rounds = (double)((tiles + pairs - 1) / pairs);
-            const double t = rounds * (kb * c.t_kb + c.epi);
+            const double t = rounds * ((kb + (lora ? lora->R / 64 : 0)) * c.t_kb + c.epi);
             if (t < best) { best = t; cfg = c.id; }
         }
     }
-#define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, Y, ldy, st
+#define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st
     switch (cfg) {
         case 1: return launch_gemm_cfg<GemmCfg<128, 1, 4, 1>>(LYNX_GEMM_ARGS);
         case 2: return launch_gemm_cfg<GemmCfg<192, 1, 3, 1>>(LYNX_GEMM_ARGS);
@@ -281,6 +305,101 @@ lynx_status ensure_scratch(lynx_ctx* ctx, size_t bytes) {
     return LYNX_OK;
 }
 
+// ----------------------------------------------------------------- low-rank down projection -----
+
+// K splits of the down projection: rounds of CTAs over the SMs x (K blocks per split + a fixed
+// per-CTA cost of ~6 K blocks for prologue and drain), smallest wins; every split is non-empty.
+void lora_split_plan(int num_sms, int64_t M, int64_t K, int* splits, int* kb_per_split) {
+    const int tiles_m = (int)((M + 127) / 128), kblocks = (int)(K / 64);
+    int best_s = 1;
+    double best = 1e30;
+    for (int sp = 1; sp <= 32 && sp * 4 <= kblocks; ++sp) {
+        const int per = (kblocks + sp - 1) / sp;
+        const int real = (kblocks + per - 1) / per;
+        const double rounds = (double)(((int64_t)tiles_m * real + num_sms - 1) / num_sms);
+        const double t = rounds * (per + 6.0);
+        if (t < best) { best = t; best_s = real; }
+    }
+    const int per = (kblocks + best_s - 1) / best_s;
+    *kb_per_split = per;
+    *splits = (kblocks + per - 1) / per;
+}
+
+struct LoraWsLayout {
+    size_t partial, T, total;
+};
+LoraWsLayout lora_ws_layout(int num_sms, int64_t M, int64_t K, int R) {
+    int splits, per;
+    lora_split_plan(num_sms, M, K, &splits, &per);
+    LoraWsLayout L;
+    const size_t tiles_m = (size_t)((M + 127) / 128);
+    L.partial = 0;
+    size_t off = align_up(splits > 1 ? tiles_m * splits * 128 * (size_t)R * 4 : 0, 1024);
+    L.T = off;
+    off = align_up(off + (size_t)M * R * 2, 1024);
+    L.total = off;
+    return L;
+}
+
+lynx_status ensure_lora_ws(lynx_ctx* ctx, size_t bytes) {
+    if (ctx->lora_ws_bytes >= bytes) return LYNX_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) return LYNX_ERR_CUDA;
+    if (ctx->lora_ws) cudaFree(ctx->lora_ws);
+    ctx->lora_ws = nullptr;
+    ctx->lora_ws_bytes = 0;
+    if (cudaMalloc(&ctx->lora_ws, bytes) != cudaSuccess) return LYNX_ERR_WORKSPACE;
+    ctx->lora_ws_bytes = bytes;
+    return LYNX_OK;
+}
+
+template <class Cfg>
+lynx_status launch_lora_down(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, const void* LB,
+                             int64_t ldlb, const float* row_scale, void* T, int64_t ldt, float* partial,
+                             cudaStream_t st) {
+    CUtensorMap tx, tlb;
+    if (!make_tmap_2d(&tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx * 2, 64,
+                      Cfg::BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tlb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, LB, (uint64_t)Cfg::R, (uint64_t)K,
+                      (uint64_t)ldlb * 2, 64, Cfg::R, CU_TENSOR_MAP_SWIZZLE_128B))
+        return LYNX_ERR_CUDA;
+    LoraDownParams p;
+    p.M = M; p.K = K;
+    lora_split_plan(ctx->num_sms, M, K, &p.splits, &p.kb_per_split);
+    p.row_scale = row_scale;
+    p.T = static_cast<uint16_t*>(T);
+    p.ldt = ldt;
+    p.partial = partial;
+    p.tickets = ctx->tickets + PRUNE_TICKET_BYTES / 4;
+    p.dev_error = ctx->err_dev;
+    auto kern = lora_down_kernel<Cfg>;
+    static bool attr_set = false;  // per instantiation
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
+            return LYNX_ERR_CUDA;
+        attr_set = true;
+    }
+    const int tiles_m = (int)((M + Cfg::BM - 1) / Cfg::BM);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(tiles_m * p.splits));
+    cfg.blockDim = dim3(Cfg::THREADS);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, tx, tlb, p) != cudaSuccess) return LYNX_ERR_CUDA;
+    ctx->launches++;
+    return LYNX_OK;
+}
+
+lynx_status check_lora_rank(int64_t R) {
+    if (R < 1) return LYNX_ERR_INVALID_ARG;
+    if (R != 64 && R != 128) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    return LYNX_OK;
+}
+
 }  // namespace
 
 // ================================================================================ C ABI ==========
@@ -307,8 +426,8 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
         return LYNX_ERR_CUDA;
     }
     *ctx->err_host = DEV_OK;
-    if (cudaMalloc(reinterpret_cast<void**>(&ctx->tickets), PRUNE_TICKET_BYTES) != cudaSuccess ||
-        cudaMemset(ctx->tickets, 0, PRUNE_TICKET_BYTES) != cudaSuccess) {
+    if (cudaMalloc(reinterpret_cast<void**>(&ctx->tickets), PRUNE_TICKET_BYTES + LORA_TICKET_BYTES) != cudaSuccess ||
+        cudaMemset(ctx->tickets, 0, PRUNE_TICKET_BYTES + LORA_TICKET_BYTES) != cudaSuccess) {
         cudaFreeHost(ctx->err_host);
         delete ctx;
         return LYNX_ERR_WORKSPACE;
@@ -331,6 +450,7 @@ lynx_status lynx_destroy(lynx_ctx* ctx) {
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->sk_partial) cudaFree(ctx->sk_partial);
     if (ctx->tickets) cudaFree(ctx->tickets);
+    if (ctx->lora_ws) cudaFree(ctx->lora_ws);
     if (ctx->err_host) cudaFreeHost(ctx->err_host);
     delete ctx;
     return LYNX_OK;
@@ -456,7 +576,8 @@ lynx_status lynx_sparse_linear(lynx_ctx* ctx, const void* values, const void* me
         if (!aligned16(comp->residual) || (comp->ldr % 8)) return LYNX_ERR_ALIGNMENT;
     }
     if ((s = check_device_error(ctx)) != LYNX_OK) return s;
-    return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, comp, Y, ldy, static_cast<cudaStream_t>(stream));
+    return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, comp, nullptr, Y, ldy,
+                       static_cast<cudaStream_t>(stream));
 }
 
 lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, const void* W,
@@ -522,6 +643,91 @@ lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_host, int64
         return LYNX_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return LYNX_ERR_CUDA;
     return check_device_error(ctx);
+}
+
+lynx_status lynx_reserve_lora(lynx_ctx* ctx, int64_t M, int64_t K, int64_t R) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if ((s = check_lora_rank(R)) != LYNX_OK) return s;
+    std::lock_guard<std::mutex> lock(ctx->mu);
+    return ensure_lora_ws(ctx, lora_ws_layout(ctx->num_sms, M, K, (int)R).total);
+}
+
+lynx_status lynx_lora_down(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, const void* LB,
+                           int64_t R, int64_t ldlb, const float* row_scale, void* T, int64_t ldt, void* stream) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if ((s = check_lora_rank(R)) != LYNX_OK) return s;
+    if (!X || !LB || !T) return LYNX_ERR_INVALID_ARG;
+    if (ldx < K || ldlb < K || ldt < R) return LYNX_ERR_INVALID_ARG;
+    if ((size_t)((M + 127) / 128) * 4 > LORA_TICKET_BYTES) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(X) || !aligned16(LB) || !aligned16(T) || (ldx % 8) || (ldlb % 8) || (ldt % 8))
+        return LYNX_ERR_ALIGNMENT;
+    if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+    const LoraWsLayout L = lora_ws_layout(ctx->num_sms, M, K, (int)R);
+    {
+        std::lock_guard<std::mutex> lock(ctx->mu);
+        if ((s = ensure_lora_ws(ctx, L.total)) != LYNX_OK) return s;
+    }
+    float* partial = reinterpret_cast<float*>(static_cast<char*>(ctx->lora_ws) + L.partial);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (R == 64) return launch_lora_down<LoraDownCfg<64>>(ctx, X, M, K, ldx, LB, ldlb, row_scale, T, ldt, partial, st);
+    return launch_lora_down<LoraDownCfg<128>>(ctx, X, M, K, ldx, LB, ldlb, row_scale, T, ldt, partial, st);
+}
+
+lynx_status lynx_sparse_linear_lora(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
+                                    const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
+                                    const void* T, int64_t ldt, const void* LA, int64_t R, int64_t ldla, void* Y,
+                                    int64_t ldy, void* stream) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if ((s = check_lora_rank(R)) != LYNX_OK) return s;
+    if (!values || !meta || !W || !Y || !T || !LA || N < 8) return LYNX_ERR_INVALID_ARG;
+    if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    if (ldw < K || ldy < N || ldt < R || ldla < R) return LYNX_ERR_INVALID_ARG;
+    if (!aligned16(values) || !aligned16(meta) || !aligned16(W) || !aligned16(Y) || !aligned16(T) || !aligned16(LA) ||
+        (ldw % 8) || (ldy % 8) || (ldt % 8) || (ldla % 8))
+        return LYNX_ERR_ALIGNMENT;
+    if (bias && !aligned16(bias)) return LYNX_ERR_ALIGNMENT;
+    if (comp && comp->residual) {
+        if (comp->ldr < N) return LYNX_ERR_INVALID_ARG;
+        if (!aligned16(comp->residual) || (comp->ldr % 8)) return LYNX_ERR_ALIGNMENT;
+    }
+    if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+    LoraArgs lora{T, ldt, LA, ldla, (int)R};
+    return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, comp, &lora, Y, ldy,
+                       static_cast<cudaStream_t>(stream));
+}
+
+lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx,
+                                        const void* W, int64_t N, int64_t ldw, const void* bias, const void* LA,
+                                        int64_t ldla, const void* LB, int64_t ldlb, int64_t R, lynx_comp_mode mode,
+                                        const void* residual, int64_t ldr, void* Y, int64_t ldy, void* stream) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if ((s = check_lora_rank(R)) != LYNX_OK) return s;
+    if (N < 8 || !LA || !LB) return LYNX_ERR_INVALID_ARG;
+    ScratchLayout L = scratch_layout(M, N, K);
+    const LoraWsLayout LL = lora_ws_layout(ctx->num_sms, M, K, (int)R);
+    {
+        std::lock_guard<std::mutex> lock(ctx->mu);
+        if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
+        if ((s = ensure_lora_ws(ctx, LL.total)) != LYNX_OK) return s;
+    }
+    char* base = static_cast<char*>(ctx->scratch);
+    void* values = base + L.values;
+    void* meta = base + L.meta;
+    float* scale = mode == LYNX_COMP_NONE ? nullptr : reinterpret_cast<float*>(base + L.scale);
+    void* T = static_cast<char*>(ctx->lora_ws) + LL.T;
+    s = lynx_prune_compress(ctx, X, M, K, ldx, values, meta, scale, mode, stream);
+    if (s != LYNX_OK) return s;
+    s = lynx_lora_down(ctx, X, M, K, ldx, LB, R, ldlb, scale, T, R, stream);
+    if (s != LYNX_OK) return s;
+    lynx_comp comp;
+    comp.row_scale = scale;
+    comp.residual = residual;
+    comp.ldr = ldr;
+    return lynx_sparse_linear_lora(ctx, values, meta, M, K, W, N, ldw, bias, &comp, T, R, LA, R, ldla, Y, ldy, stream);
 }
 
 lynx_status lynx_meta_to_canonical(lynx_ctx* ctx, const void* meta, int64_t M, int64_t K, void* meta_canon,

@@ -270,6 +270,27 @@ __device__ __forceinline__ void mma_sp_bf16_lh(uint32_t d_tmem, uint32_t a_lo, u
             : "memory");
 }
 
+// Dense form (no metadata operand): D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> fp32, K = 16
+// per instruction.  Same descriptor convention as mma_sp_bf16_lh.
+template <int CG>
+__device__ __forceinline__ void mma_bf16_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                            uint32_t idesc, uint32_t accumulate) {
+    if constexpr (CG == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem),
+            "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem),
+            "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+}
+
 // 128 lanes x 128 bits, shared memory -> tensor memory (4 columns).
 template <int CG>
 __device__ __forceinline__ void tmem_cp_128x128b(uint32_t taddr, uint64_t s_desc) {

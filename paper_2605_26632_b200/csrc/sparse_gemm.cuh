@@ -15,6 +15,12 @@
 //               TMA-store 32 x 64 boxes
 // With two accumulator buffers the epilogue of tile i overlaps the main loop of tile i+1.
 //
+// Low-rank branch (Algorithm 1 lines 5-6, Y = Y_s + X (L_A L_B)^T): when lora_steps > 0 every
+// tile gets lora_steps extra ring stages after its last K block.  Such a stage holds a 128 x 64
+// box of T = (X L_B^T) / s (bf16, produced by lora_down_kernel) in the A slot and a BN x 64 box of
+// L_A in the W slot, and the issuer adds T L_A^T with four DENSE tcgen05.mma (K = 16 each) into
+// the same accumulator, so Y_r never exists in memory and the epilogue's s_m * acc restores it.
+//
 // CG == 2: the pair computes a 256 x BN tile; each CTA stages its own 128 rows of A and
 // metadata and its own BN/2 rows of W (plain TMA loads, no multicast), the leader CTA issues
 // cta_group::2 MMAs, and each CTA drains its own 128 accumulator rows.
@@ -37,6 +43,7 @@ struct GemmParams {
     float* sk_partial;
     uint32_t* sk_flags;
     uint32_t sk_epoch;
+    int lora_steps;  // R / 64 extra dense stages per tile (0 = no low-rank branch)
 };
 
 // Work distribution over C persistent clusters.  The first floor(T/C)*C tiles go round-robin,
@@ -135,7 +142,7 @@ struct GemmCfg {
 };
 
 // Instruction descriptor of tcgen05.mma.sp kind::f16: bf16 x bf16 -> fp32, both operands
-// K-major, sparse, M x N per instruction.
+// K-major, sparse, M x N per instruction (clearing bit 2 gives the dense instruction's).
 __host__ __device__ constexpr uint32_t make_idesc_sp_bf16(int m, int n) {
     return (1u << 2)                        // sparse
            | (1u << 4)                      // D format: fp32
@@ -149,6 +156,7 @@ template <class Cfg>
 __global__ void __launch_bounds__(Cfg::THREADS, 1)
 sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                    const __grid_constant__ CUtensorMap tmap_e, const __grid_constant__ CUtensorMap tmap_y,
+                   const __grid_constant__ CUtensorMap tmap_t, const __grid_constant__ CUtensorMap tmap_la,
                    const GemmParams p) {
     constexpr int CG = Cfg::CG, STAGES = Cfg::STAGES, BN = Cfg::BN;
     extern __shared__ uint8_t smem_raw[];
@@ -189,6 +197,10 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         prefetch_tmap(&tmap_b);
         prefetch_tmap(&tmap_e);
         prefetch_tmap(&tmap_y);
+        if (p.lora_steps) {
+            prefetch_tmap(&tmap_t);
+            prefetch_tmap(&tmap_la);
+        }
     }
     if (warp == 1) {
         tmem_alloc<CG>(smem_u32(tmem_slot), Cfg::TMEM_COLS);
@@ -243,6 +255,31 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
+                // low-rank stages: T box in the A slot, L_A box in the first half of the W slot
+                if (w.kb1 == kblocks) {
+                    for (int j = 0; j < p.lora_steps && ok; ++j) {
+                        if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, cta_abort, p.dev_error)) {
+                            ok = false;
+                            break;
+                        }
+                        constexpr uint32_t LORA_BYTES = Cfg::A_BYTES + Cfg::B_HALF_BYTES;
+                        const uint32_t a_dst = sA + stage * Cfg::A_BYTES;
+                        const uint32_t b_dst = sB + stage * Cfg::B_BYTES;
+                        if constexpr (CG == 1) {
+                            const uint32_t bar = bar_full + 8 * stage;
+                            mbar_arrive_expect_tx(bar, LORA_BYTES);
+                            tma_load_2d(a_dst, &tmap_t, j * 64, m0, bar);
+                            tma_load_2d(b_dst, &tmap_la, j * 64, n0, bar);
+                        } else {
+                            const uint32_t bar = full0 + 8 * stage;
+                            if (leader) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * LORA_BYTES);
+                            tma_load_2d_pair(a_dst, &tmap_t, j * 64, m0, bar);
+                            tma_load_2d_pair(b_dst, &tmap_la, j * 64, n0, bar);
+                        }
+                        ++issued;
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    }
+                }
             }
             if (!ok && issued) bounded_delay_ns(200000);  // let the copies in flight land before teardown
         }
@@ -288,6 +325,27 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     else tc_commit_pair(bar_empty + 8 * stage, 0x3);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
+                if (ok && w.kb1 == kblocks) {
+                    constexpr uint32_t idesc_dense = idesc0 & ~(1u << 2);
+                    for (int j = 0; j < p.lora_steps; ++j) {
+                        if (!mbar_wait(bar_full + 8 * stage, phase, cta_abort, p.dev_error)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t a_lo = a_lo0 + stage * (Cfg::A_BYTES >> 4);
+                        const uint32_t b_lo = b_lo0 + stage * (Cfg::B_BYTES >> 4);
+                        // dense K steps of 16 elements: both operands advance 32 bytes
+                        mma_bf16_lh<CG>(d_tmem, a_lo, b_lo, desc_hi, idesc_dense, accumulate);
+                        mma_bf16_lh<CG>(d_tmem, a_lo + 2, b_lo + 2, desc_hi, idesc_dense, 1u);
+                        mma_bf16_lh<CG>(d_tmem, a_lo + 4, b_lo + 4, desc_hi, idesc_dense, 1u);
+                        mma_bf16_lh<CG>(d_tmem, a_lo + 6, b_lo + 6, desc_hi, idesc_dense, 1u);
+                        accumulate = 1u;
+                        if constexpr (CG == 1) tc_commit(bar_empty + 8 * stage);
+                        else tc_commit_pair(bar_empty + 8 * stage, 0x3);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    }
+                }
                 if (!ok) break;
                 if constexpr (CG == 1) tc_commit(bar_tfull + 8 * acc);
                 else tc_commit_pair(bar_tfull + 8 * acc, 0x3);
@@ -329,8 +387,8 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
                 if (!alive) break;
             }
-#pragma unroll 1
             constexpr int CH = Cfg::CH;
+#pragma unroll 1
             for (int c = 0; c < BN / CH; ++c) {
                 const int n0 = tn * BN + c * CH;
                 uint32_t v[CH];

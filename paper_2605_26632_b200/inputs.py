@@ -100,6 +100,15 @@ def make_residual(M: int, N: int, seed: int) -> torch.Tensor:
     return (torch.randn(M, N, generator=g, dtype=torch.float32) * 0.05).to(torch.bfloat16).contiguous()
 
 
+def make_lora(N: int, K: int, R: int, seed: int):
+    """Low-rank factors -> (L_A [N, R], L_B [R, K]) bf16: L_B ~ N(0, 1/K), L_A ~ N(0, 0.3^2 / R),
+    so that X (L_A L_B)^T is a correction of about a third of the main product's magnitude."""
+    g = _gen(seed + 4_000_003)
+    lb = torch.randn(R, K, generator=g, dtype=torch.float32) * (K ** -0.5)
+    la = torch.randn(N, R, generator=g, dtype=torch.float32) * (0.3 * R ** -0.5)
+    return la.to(torch.bfloat16).contiguous(), lb.to(torch.bfloat16).contiguous()
+
+
 def make_workload(w: Workload, with_bias: bool = True, with_residual: bool = False,
                   M: Optional[int] = None):
     """-> dict(X, W, bias, residual) of CPU bf16 tensors (bias/residual may be None)."""

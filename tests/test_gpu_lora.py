@@ -1,0 +1,201 @@
+"""GPU parity tests of the low-rank branch (Algorithm 1 lines 5-6, Y = Y_s + X (L_A L_B)^T):
+down projection kernel, the dense accumulator steps inside the sparse GEMM, and the whole layer,
+through the C ABI against the CPU oracle.
+
+Bars: T = bf16((X L_B^T) / s) within one bf16 rounding (2^-8 relative) plus the fp32
+summation-order slack of the oracle's fp32 result; Y within relative Frobenius error 5e-3 and
+max |dY| <= 2e-2 * max |Y_ref| (the T rounding is of the same size as Y's own bf16 rounding).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_26632_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+RFE_TOL = 5e-3
+MAXABS_TOL = 2e-2
+
+
+@pytest.fixture(scope="module")
+def lx():
+    from paper_2605_26632_b200 import binding
+
+    ctx = binding.Lynx(0)
+    yield ctx
+    torch.cuda.synchronize()
+    assert ctx.last_error() == 0
+    ctx.close()
+
+
+def u16(t):
+    return inputs.as_u16(t.detach().cpu())
+
+
+def check_y(Y, ref):
+    yf = Y.float().cpu().numpy()
+    rfe = np.linalg.norm(yf - ref) / max(np.linalg.norm(ref), 1e-30)
+    mx = np.abs(yf - ref).max() / max(np.abs(ref).max(), 1e-30)
+    assert rfe <= RFE_TOL, f"relative Frobenius error {rfe}"
+    assert mx <= MAXABS_TOL, f"max abs error ratio {mx}"
+
+
+def make_case(M, K, N, R, seed, dist="outlier", with_bias=True, with_res=False):
+    X = inputs.make_x(M, K, dist, seed)
+    W = inputs.make_w(N, K, seed)
+    b = inputs.make_bias(N, seed) if with_bias else None
+    res = inputs.make_residual(M, N, seed) if with_res else None
+    LA, LB = inputs.make_lora(N, K, R, seed)
+    return X, W, b, res, LA, LB
+
+
+def oracle_t(X, LB, mode):
+    """(X L_B^T) / s from the oracle: the residual through an identity L_A is the down projection."""
+    R = LB.shape[0]
+    eye = torch.eye(R, dtype=torch.bfloat16)
+    t = oracle.lora_residual(u16(X), u16(LB), u16(eye))
+    if mode:
+        s = oracle.row_scale(u16(X), mode).astype(np.float32)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            t = np.where(s[:, None] == 0, 0.0, t / s[:, None]).astype(np.float32)
+    return t
+
+
+@pytest.mark.parametrize("M,K,R,mode", [
+    (256, 512, 64, 0), (256, 512, 64, 1), (300, 1024, 64, 1), (129, 128, 64, 2), (1000, 3072, 128, 1),
+    (4096, 3072, 64, 1), (2048, 12288, 64, 1),
+])
+def test_lora_down_matches_oracle(lx, M, K, R, mode):
+    X = inputs.make_x(M, K, "outlier", 40 + M)
+    _, LB = inputs.make_lora(8, K, R, 41 + M)
+    Xc = X.cuda()
+    scale = None
+    if mode:
+        _, _, scale = lx.prune_compress(Xc, mode)
+    T = lx.lora_down(Xc, LB.cuda(), scale)
+    ref = oracle_t(X, LB, mode)
+    got = T.float().cpu().numpy()
+    tol = 2.0 ** -8 * np.abs(ref) + 1e-5 * np.abs(ref).max()
+    assert (np.abs(got - ref) <= tol).all(), float(np.abs(got - ref).max())
+    # reproducible whichever CTA finishes last
+    T2 = lx.lora_down(Xc, LB.cuda(), scale)
+    assert torch.equal(T, T2)
+
+
+def test_lora_down_zero_rows_and_strided_output(lx):
+    M, K, R = 200, 256, 64
+    X = inputs.make_x(M, K, "outlier", 7)
+    X[5] = 0
+    X[199] = 0
+    _, LB = inputs.make_lora(8, K, R, 7)
+    Xc = X.cuda()
+    _, _, scale = lx.prune_compress(Xc, 1)
+    buf = torch.full((M, 2 * R), 7.0, dtype=torch.bfloat16, device="cuda")
+    T = lx.lora_down(Xc, LB.cuda(), scale, out=buf[:, :R])
+    assert (T[5] == 0).all() and (T[199] == 0).all()
+    assert (buf[:, R:] == 7.0).all()
+    ref = oracle_t(X, LB, 1)
+    assert np.abs(T.float().cpu().numpy() - ref).max() <= 2.0 ** -8 * np.abs(ref).max() + 1e-6
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("with_bias,with_res", [(False, False), (True, True)])
+def test_tiny_config_with_lora_full_oracle(lx, mode, with_bias, with_res):
+    wl = inputs.WORKLOADS["tiny"]
+    X, W, b, res, LA, LB = make_case(wl.M, wl.K, wl.N, 64, wl.seed, wl.x_dist, with_bias, with_res)
+    ref = oracle.act_sparse_linear_lora(u16(X), u16(W), u16(LA), u16(LB), bias=None if b is None else u16(b),
+                                        comp_mode=mode, Yr=None if res is None else u16(res))
+    cu = lambda t: None if t is None else t.cuda()
+    Y = lx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), cu(b), mode, cu(res))
+    check_y(Y, ref["Y"])
+    # the three-call form gives the same bits
+    values, meta, scale = lx.prune_compress(X.cuda(), mode)
+    T = lx.lora_down(X.cuda(), LB.cuda(), scale)
+    Y2 = lx.sparse_linear_lora(values, meta, W.cuda(), T, LA.cuda(), cu(b), scale, cu(res))
+    assert torch.equal(Y, Y2)
+    # and the branch really contributes: without it the result is off by the residual's size
+    Y0 = lx.act_sparse_linear(X.cuda(), W.cuda(), cu(b), mode, cu(res))
+    assert (Y.float() - Y0.float()).abs().max().item() > 0.05
+
+
+def test_zero_weight_leaves_the_dense_low_rank_product(lx):
+    """W = 0: Y must equal X (L_A L_B)^T computed from the DENSE X (silicon check of the dense
+    tensor-core steps: operand order, K advance, both halves of a CTA pair)."""
+    M, K, N, R = 520, 384, 1000, 64
+    X, _, _, _, LA, LB = make_case(M, K, N, R, 77)
+    W = torch.zeros(N, K, dtype=torch.bfloat16)
+    Y = lx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), None, 1)
+    ref = ((X.double() @ LB.double().T) @ LA.double().T).numpy()
+    check_y(Y, ref)
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6, 7])
+@pytest.mark.parametrize("R", [64, 128])
+def test_every_tile_configuration_with_lora(cfg, R, monkeypatch):
+    from paper_2605_26632_b200 import binding
+
+    monkeypatch.setenv("LYNX_GEMM_CFG", str(cfg))
+    ctx = binding.Lynx(0)
+    try:
+        M, K, N = 700, 640, 1096  # ragged in M and N for every tile width
+        X, W, b, res, LA, LB = make_case(M, K, N, R, 500 + cfg, with_res=True)
+        ref = oracle.act_sparse_linear_lora(u16(X), u16(W), u16(LA), u16(LB), bias=u16(b), comp_mode=1, Yr=u16(res))
+        Y = ctx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), b.cuda(), 1, res.cuda())
+        check_y(Y, ref["Y"])
+        Y2 = ctx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), b.cuda(), 1, res.cuda())
+        assert torch.equal(Y, Y2)
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
+
+
+@pytest.mark.parametrize("cfg", [4, 7])
+def test_stream_k_with_lora(cfg, monkeypatch):
+    from paper_2605_26632_b200 import binding
+
+    monkeypatch.setenv("LYNX_GEMM_CFG", str(cfg))
+    monkeypatch.setenv("LYNX_STREAMK", "1")
+    ctx = binding.Lynx(0)
+    try:
+        M, K, N = 2304, 2048, 2880  # leaves a tail of tiles, long enough in K for the stream-K split
+        X, W, b, _, LA, LB = make_case(M, K, N, 64, 600 + cfg)
+        rows = np.arange(0, M, 37, dtype=np.int64)
+        ref = oracle.act_sparse_linear_lora(u16(X), u16(W), u16(LA), u16(LB), bias=u16(b), comp_mode=1, rows=rows)
+        Y = ctx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), b.cuda(), 1)
+        check_y(Y[torch.from_numpy(rows).cuda()], ref["Y"])
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
+
+
+@pytest.mark.parametrize("name", ["mlp_down", "attn_out", "mlp_up"])
+def test_dit_workloads_full_size_with_lora(lx, name):
+    wl = inputs.WORKLOADS[name]
+    X, W, b, _, LA, LB = make_case(wl.M, wl.K, wl.N, 64, wl.seed, wl.x_dist)
+    rows = np.sort(np.random.default_rng(wl.seed).choice(wl.M, 24, replace=False)).astype(np.int64)
+    rows[0], rows[-1] = 0, wl.M - 1
+    ref = oracle.act_sparse_linear_lora(u16(X), u16(W), u16(LA), u16(LB), bias=u16(b), comp_mode=1, rows=rows)
+    Y = lx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), b.cuda(), 1)
+    check_y(Y[torch.from_numpy(rows).cuda()], ref["Y"])
+
+
+def test_lora_argument_errors(lx):
+    from paper_2605_26632_b200.binding import LynxError
+
+    X = torch.zeros(128, 256, dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros(64, 256, dtype=torch.bfloat16, device="cuda")
+    for R in (32, 96, 256):
+        LA = torch.zeros(64, R, dtype=torch.bfloat16, device="cuda")
+        LB = torch.zeros(R, 256, dtype=torch.bfloat16, device="cuda")
+        n0 = lx.launch_count()
+        with pytest.raises(LynxError) as e:
+            lx.act_sparse_linear_lora(X, W, LA, LB)
+        assert e.value.status == 2  # unsupported shape
+        assert lx.launch_count() == n0
+    LB = torch.zeros(64, 512, dtype=torch.bfloat16, device="cuda")[:, ::2]  # wrong inner stride
+    with pytest.raises(TypeError):
+        lx.lora_down(X, LB)
