@@ -193,27 +193,52 @@ lora_down_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             asm volatile("bar.sync 1, 128;" ::: "memory");
             // a CTA that timed out still takes its ticket (so nobody is left waiting); the error
             // word tells the host that T is not valid
-            if (*s_last && row_ok) {
-                float s = 1.0f;
-                if (p.row_scale != nullptr) s = p.row_scale[row];
-                const float* src0 = p.partial + ((size_t)tm * p.splits * Cfg::BM + r_in_tile) * R;
+            if (*s_last) {
+                // 128 threads x 8-column pieces, consecutive threads on consecutive pieces; four
+                // pieces at a time so that 8 * (splits unrolled by 2) loads are in flight per thread
+                const int t = threadIdx.x - 64;
+                constexpr int PIECES_PER_ROW = R / 8;
+                constexpr int ITEMS = Cfg::BM * PIECES_PER_ROW / 128;
+                const float* base = p.partial + (size_t)tm * p.splits * Cfg::BM * R;
 #pragma unroll 1
-                for (int c = 0; c < R / 8; ++c) {
-                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                    for (int sp = 0; sp < p.splits; ++sp) {  // ascending split order, always
-                        const float4* src = reinterpret_cast<const float4*>(src0 + (size_t)sp * Cfg::BM * R + c * 8);
-                        const float4 a = __ldcg(src), b = __ldcg(src + 1);
-                        acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
-                        acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
-                    }
-                    uint32_t o[4];
+                for (int i0 = 0; i0 < ITEMS; i0 += 4) {
+                    float acc[4][8];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float t0 = (s == 0.0f) ? 0.0f : __fdiv_rn(acc[2 * e], s);
-                        const float t1 = (s == 0.0f) ? 0.0f : __fdiv_rn(acc[2 * e + 1], s);
-                        o[e] = pack_bf16x2(t0, t1);
+                    for (int u = 0; u < 4; ++u)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[u][e] = 0.0f;
+#pragma unroll 2
+                    for (int sp = 0; sp < p.splits; ++sp) {  // ascending split order, always
+                        float4 a[4], b[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int idx = (i0 + u) * 128 + t;  // = row * PIECES_PER_ROW + piece
+                            const float4* src = reinterpret_cast<const float4*>(base + (size_t)sp * Cfg::BM * R + (size_t)idx * 8);
+                            a[u] = __ldcg(src);
+                            b[u] = __ldcg(src + 1);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            acc[u][0] += a[u].x; acc[u][1] += a[u].y; acc[u][2] += a[u].z; acc[u][3] += a[u].w;
+                            acc[u][4] += b[u].x; acc[u][5] += b[u].y; acc[u][6] += b[u].z; acc[u][7] += b[u].w;
+                        }
                     }
-                    *reinterpret_cast<uint4*>(p.T + row * p.ldt + c * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int idx = (i0 + u) * 128 + t;
+                        const int r_t = idx / PIECES_PER_ROW, piece = idx % PIECES_PER_ROW;
+                        const int64_t grow = (int64_t)tm * Cfg::BM + r_t;
+                        if (grow >= p.M) continue;
+                        const float s = (p.row_scale != nullptr) ? p.row_scale[grow] : 1.0f;
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float t0 = (s == 0.0f) ? 0.0f : __fdiv_rn(acc[u][2 * e], s);
+                            const float t1 = (s == 0.0f) ? 0.0f : __fdiv_rn(acc[u][2 * e + 1], s);
+                            o[e] = pack_bf16x2(t0, t1);
+                        }
+                        *reinterpret_cast<uint4*>(p.T + grow * p.ldt + piece * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
                 }
             }
         }

@@ -1,6 +1,6 @@
 """Runs a few launches of one kernel of the path on a named synthetic workload.
 
-    python -m paper_2605_26632_b200.run_case --kernel prune|gemm|layer|fused --workload mlp_down [--iters 3]
+    python -m paper_2605_26632_b200.run_case --kernel prune|gemm|layer|fused|lora_down|lora_layer --workload mlp_down [--iters 3]
 
 Meant as the small, self-terminating command to put under a profiler (one kernel, a few launches,
 well under a GB on the device), and as a minimal usage example of the binding.
@@ -16,7 +16,8 @@ from . import binding, inputs
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="layer", choices=["prune", "gemm", "layer", "fused"])
+    ap.add_argument("--kernel", default="layer", choices=["prune", "gemm", "layer", "fused", "lora_down", "lora_layer"])
+    ap.add_argument("--rank", type=int, default=64, help="rank R of the low-rank branch")
     ap.add_argument("--workload", default="mlp_down")
     ap.add_argument("--M", type=int, default=0, help="override the number of token rows")
     ap.add_argument("--iters", type=int, default=3)
@@ -33,11 +34,21 @@ def main():
     lx.reserve(M, wl.N, wl.K)
     values, meta, scale = lx.prune_compress(X, args.comp)
     Y = torch.empty(M, wl.N, device="cuda", dtype=torch.bfloat16)
+    R = args.rank
+    LB = (torch.randn(R, wl.K, device="cuda", generator=g) * wl.K ** -0.5).to(torch.bfloat16)
+    LA = (torch.randn(wl.N, R, device="cuda", generator=g) * 0.3 * R ** -0.5).to(torch.bfloat16)
+    T = torch.empty(M, R, device="cuda", dtype=torch.bfloat16)
+    if args.kernel.startswith("lora"):
+        lx.reserve_lora(M, wl.K, R)
     for _ in range(args.iters):
         if args.kernel in ("prune", "layer"):
             lx.prune_compress(X, args.comp, values, meta, scale)
         if args.kernel in ("gemm", "layer"):
             lx.sparse_linear(values, meta, W, b, scale, None, Y)
+        if args.kernel == "lora_down":
+            lx.lora_down(X, LB, scale, T)
+        if args.kernel == "lora_layer":
+            lx.act_sparse_linear_lora(X, W, LA, LB, b, args.comp, None, Y)
         if args.kernel == "fused":
             lx.act_sparse_linear(X, W, b, args.comp, None, Y, binding.FUSE_FUSED)
     torch.cuda.synchronize()

@@ -5,7 +5,8 @@
 For each (M, K, N): prune/compress alone (GB/s of its 3.125 B/element), sparse GEMM alone, the
 two-kernel layer, the fused one-kernel layer, and the dense bf16 linear (torch / cuBLASLt) on the
 same GPU with the same timing loop.  Inputs rotate over enough copies that nothing a launch reads
-is left in the L2 by the previous launch; times are CUDA-event averages over `iters` launches.
+is left in the L2 by the previous launch; times are CUDA-event averages over `iters` launches
+replayed from a CUDA graph (`--no-graph`: eager launches, host-bound below ~15 us per call).
 """
 from __future__ import annotations
 
@@ -17,17 +18,37 @@ import torch
 from . import binding, inputs
 
 
+USE_GRAPH = True
+
+
 def timeloop(fn, nsets, iters, warm=5):
+    """Average device time of one call of fn (ms).  The `iters` calls are captured into one CUDA
+    graph and the graph is replayed, so that launches shorter than the host's per-call cost
+    (tensor-map encoding + launch, ~10 us from Python) are timed at the GPU's pace, not the host's."""
     for i in range(warm):
         fn(i % nsets)
     torch.cuda.synchronize()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if not USE_GRAPH:
+        a.record()
+        for i in range(iters):
+            fn(i % nsets)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(iters):
+            fn(i % nsets)
+    g.replay()
+    torch.cuda.synchronize()
+    reps = 3
     a.record()
-    for i in range(iters):
-        fn(i % nsets)
+    for _ in range(reps):
+        g.replay()
     b.record()
     torch.cuda.synchronize()
-    return a.elapsed_time(b) / iters  # ms
+    return a.elapsed_time(b) / (iters * reps)
 
 
 def main():
@@ -35,7 +56,13 @@ def main():
     ap.add_argument("--quick", action="store_true", help="M = 4096 only")
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--no-fused", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph replay")
+    ap.add_argument("--lora", type=int, default=0, metavar="R",
+                    help="time the low-rank branch of rank R instead: down projection alone, layer with it, "
+                         "and the dense linear followed by the two dense low-rank GEMMs of torch")
     args = ap.parse_args()
+    global USE_GRAPH
+    USE_GRAPH = not args.no_graph
     lx = binding.Lynx(0)
     Ms = (4096,) if args.quick else inputs.SWEEP_M
     shapes = [(M, K, N) for M in Ms for (K, N) in inputs.SWEEP_KN]
@@ -43,6 +70,8 @@ def main():
     shapes += [(inputs.OTHER_FAMILY_M, K, N) for (K, N) in inputs.OTHER_FAMILY_KN]
     if not args.quick:
         shapes += [(M, K, M) for M in (2048, 4096, 8192) for K in (3072, 12288)]  # the paper's kernel grid
+    if args.lora:
+        return lora_sweep(lx, shapes, args.lora, args.iters)
     print("| M | K | N | prune us | prune GB/s | GEMM us | GEMM TF | layer us | layer TF | fused us | fused TF | "
           "dense us | dense TF | GEMM/dense | layer/dense |")
     print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
@@ -75,6 +104,40 @@ def main():
               f"{td/tg:.2f} | {td/tl:.2f} |", flush=True)
         assert lx.last_error() == 0
         del Xs, Ws, vs, ms, ss, Ys
+        torch.cuda.empty_cache()
+
+
+def lora_sweep(lx, shapes, R, iters):
+    print("| M | K | N | R | lora_down us | lora_down GB/s | layer us | layer+LoRA us | overhead | "
+          "dense+LoRA (torch) us | speedup with LoRA |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|")
+    for (M, K, N) in shapes:
+        per_set = M * K * 2 + M * K + M * K // 8 + N * K * 2 + M * N * 2
+        nsets = max(2, math.ceil(400e6 / per_set))
+        g = torch.Generator(device="cuda").manual_seed(M + K + N)
+        Xs = [torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16) for _ in range(nsets)]
+        Ws = [(torch.randn(N, K, device="cuda", generator=g) * K ** -0.5).to(torch.bfloat16) for _ in range(nsets)]
+        LB = (torch.randn(R, K, device="cuda", generator=g) * K ** -0.5).to(torch.bfloat16)
+        LA = (torch.randn(N, R, device="cuda", generator=g) * 0.3 * R ** -0.5).to(torch.bfloat16)
+        b = torch.zeros(N, device="cuda", dtype=torch.bfloat16)
+        Ys = [torch.empty(M, N, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+        Ts = [torch.empty(M, R, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+        ss = [torch.ones(M, device="cuda", dtype=torch.float32) for _ in range(nsets)]
+        lx.reserve(M, N, K)
+        lx.reserve_lora(M, K, R)
+        td = timeloop(lambda j: lx.lora_down(Xs[j], LB, ss[j], Ts[j]), nsets, iters)
+        tl = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_SEPARATE), nsets, iters)
+        tll = timeloop(lambda j: lx.act_sparse_linear_lora(Xs[j], Ws[j], LA, LB, b, 1, None, Ys[j]), nsets, iters)
+
+        def dense_lora(j):
+            y = torch.nn.functional.linear(Xs[j], Ws[j], b)
+            y.addmm_(torch.nn.functional.linear(Xs[j], LB), LA.t())
+
+        tdl = timeloop(dense_lora, nsets, iters)
+        print(f"| {M} | {K} | {N} | {R} | {td*1e3:.1f} | {M*K*2/td/1e6:.0f} | {tl*1e3:.1f} | {tll*1e3:.1f} | "
+              f"{100*(tll/tl-1):.1f} % | {tdl*1e3:.1f} | {tdl/tll:.2f} |", flush=True)
+        assert lx.last_error() == 0
+        del Xs, Ws, Ys, Ts, ss
         torch.cuda.empty_cache()
 
 
