@@ -25,8 +25,12 @@ struct lynx_ctx {
     void* scratch = nullptr;  // compressed operands, scale, sums, host staging mirrors
     size_t scratch_bytes = 0;
     uint32_t* tickets = nullptr;  // one word per 16-row block (prune finalize), zero between launches
-    void* lora_ws = nullptr;      // low-rank branch: [fp32 partials of the down projection][T]
+    void* lora_ws = nullptr;      // low-rank branch: [fp32 partials][T]
     size_t lora_ws_bytes = 0;
+    uint32_t l0_epoch = 0;        // launch counter of the fused down projection (ready words hold it)
+    uint32_t l0_done_total = 0;   // groups published by all such launches so far (mod 2^32)
+    int l0_force_splits = 0, l0_force_fill = -1;  // development overrides of the phase-0 plan
+    int lora_fuse = 1;            // down projection inside the GEMM launch when the tile allows (LYNX_LORA_FUSE=0: own kernel)
     float* sk_partial = nullptr;  // stream-K partial tiles (one slot per cluster) + ready words
     uint32_t* sk_flags = nullptr;
     uint32_t sk_epoch = 0;
@@ -86,6 +90,10 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 constexpr size_t PRUNE_TICKET_BYTES = 1u << 20;  // 262144 row blocks of 16 rows = 4M rows
 constexpr size_t LORA_TICKET_BYTES = 64u << 10;  // after the prune tickets: 16384 row blocks of 128 rows
+// in-GEMM down projection: ticket and ready word per 32-row group (65536 groups = 2M rows), each
+// at a fixed place of the zero-initialised ticket allocation, whatever shapes the context serves
+constexpr size_t L0_WORDS_BYTES = 256u << 10;
+constexpr size_t TICKET_ALLOC_BYTES = PRUNE_TICKET_BYTES + LORA_TICKET_BYTES + 2 * L0_WORDS_BYTES + 256;  // + done counter
 
 // Low-rank branch operands of the GEMM: T = (X L_B^T) / s [M x R] bf16 and L_A [N x R] bf16.
 struct LoraArgs {
@@ -94,7 +102,59 @@ struct LoraArgs {
     const void* LA;
     int64_t ldla;
     int R;
+    // set when the GEMM launch computes T itself (phase 0): dense X, L_B and the workspace pieces
+    const void* X = nullptr;
+    int64_t ldx = 0;
+    const void* LB = nullptr;
+    int64_t ldlb = 0;
+    float* l0_partial = nullptr;
+    uint32_t* l0_tickets = nullptr;
+    uint32_t* l0_ready = nullptr;
 };
+
+// Plan of the in-GEMM down projection: items = 256-row blocks x K splits.  Clusters with one tile
+// fewer than the busiest ("light": index >= tiles % clusters) have a tile time of slack.  If ALL
+// items fit into that slack (at most `fill` per light cluster) they go there and the busiest
+// clusters carry none; otherwise every cluster takes its share round-robin, which finishes T
+// soonest -- a T that is late stalls the first tile of every cluster at its low-rank stage
+// (measured: a partial placement on few light clusters cost more than it saved).
+// t_tile_us: one tile's main loop; an item streams its K blocks at about 0.75 us per 128-element
+// block while most clusters stream too (HBM bound), plus ~1 us of pipeline fill.
+struct L0Plan {
+    int splits, kb_per_split, light0, fill;
+};
+L0Plan l0_plan(int clusters, int tiles, int tiles_m, int kblocks, double t_tile_us, int force_splits, int force_fill) {
+    L0Plan best{1, kblocks, clusters, 0};
+    double best_t = 1e30;
+    const int rem = tiles % clusters, light = rem ? clusters - rem : 0;
+    for (int sp = 1; sp <= 16 && (sp == 1 || sp * 2 <= kblocks); ++sp) {
+        if (force_splits > 0 && sp != force_splits) continue;
+        const int per = (kblocks + sp - 1) / sp;
+        const int real = (kblocks + per - 1) / per;
+        const int items = tiles_m * real;
+        // finalize: one L2 round trip per split under load, plus fences and the ticket
+        const double t_fin = real > 1 ? 1.5 + 1.3 * real : 0.5;
+        // inside the slack of the light clusters: few clusters stream, ~0.42 us per K block
+        const double t_item_s = per * 0.42 + 2.0;
+        int fill = light ? (int)((t_tile_us - t_fin) / t_item_s) : 0;
+        if (fill > 8) fill = 8;
+        if (fill < 0) fill = 0;
+        if (force_fill >= 0) fill = light ? force_fill : 0;
+        if (fill > 0 && light * fill >= items) {
+            const double t = 0.02 * real;
+            if (t < best_t) { best_t = t; best = L0Plan{real, per, rem, fill}; }
+        }
+        if (force_fill > 0) continue;
+        // round-robin over all clusters: everybody streams, ~0.75 us per K block
+        const double t_item_r = per * 0.75 + 1.0;
+        const double late = t_fin - 0.5 * t_tile_us;
+        const double t = (double)((items + clusters - 1) / clusters) * t_item_r + (late > 0 ? late : 0) + 0.02 * real;
+        if (t < best_t) { best_t = t; best = L0Plan{real, per, clusters, 0}; }
+    }
+    return best;
+}
+// upper bound of the splits any plan uses (workspace sizing)
+constexpr int L0_MAX_SPLITS = 16;
 
 // Scratch layout for (M, N, K):
 // [partial row sums][sums 2M floats][values][meta][row_scale M floats][X stage][Y stage]
@@ -125,7 +185,7 @@ template <class Cfg>
 lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
                             const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
                             const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st) {
-    CUtensorMap ta, tb, te, ty, tt, tla;
+    CUtensorMap ta, tb, te, ty, tt, tla, tx, tlb;
     const uint64_t rb = (uint64_t)((M + 127) / 128), kblocks = (uint64_t)(K / 128);
     if (!make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, values, (uint64_t)M, (uint64_t)(K / 2),
                       (uint64_t)K, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
@@ -146,6 +206,18 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
         tt = ta;  // never read: lora_steps = 0
         tla = tb;
     }
+    const bool l0 = lora && lora->X && Cfg::L0_OK && lora->R == Cfg::L0_R;
+    if (lora && lora->X && !l0) return LYNX_ERR_INVALID_ARG;  // the caller checks the tile first
+    if (l0) {
+        if (!make_tmap_2d(&tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->X, (uint64_t)M, (uint64_t)K,
+                          (uint64_t)lora->ldx * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap_2d(&tlb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->LB, (uint64_t)lora->R, (uint64_t)K,
+                          (uint64_t)lora->ldlb * 2, 64, Cfg::L0_R / Cfg::CG, CU_TENSOR_MAP_SWIZZLE_128B))
+            return LYNX_ERR_CUDA;
+    } else {
+        tx = ta;
+        tlb = tb;
+    }
 
     GemmParams p;
     p.lora_steps = lora ? lora->R / 64 : 0;
@@ -160,6 +232,19 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     p.sk_partial = nullptr;
     p.sk_flags = nullptr;
     p.sk_epoch = 0;
+    p.l0_fused = l0 ? 1 : 0;
+    p.l0_splits = 1;
+    p.l0_kb_per_split = 0;
+    p.l0_light0 = 0;
+    p.l0_fill = 0;
+    p.l0_partial = nullptr;
+    p.l0_tickets = nullptr;
+    p.l0_ready = nullptr;
+    p.l0_epoch = 0;
+    p.l0_done = nullptr;
+    p.l0_done_target = 0;
+    p.T = nullptr;
+    p.ldt = 0;
 
     auto kern = sparse_gemm_kernel<Cfg>;
     static bool attr_set = false;  // per instantiation
@@ -175,7 +260,7 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
         // at least 4 blocks; needs the per-cluster partial slots (allocated once, on first use)
         const int kblocks = (int)(K / Cfg::BK);
         const int rem = tiles % clusters;
-        if (ctx->streamk && rem > 0 && (int64_t)rem * kblocks >= 4ll * clusters) {
+        if (!l0 && ctx->streamk && rem > 0 && (int64_t)rem * kblocks >= 4ll * clusters) {
             if (!ctx->sk_partial) {
                 const size_t slot = (size_t)128 * 256 * 4, nslots = (size_t)ctx->num_sms;
                 void* buf = nullptr;
@@ -190,6 +275,24 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
         } else if (clusters > tiles) {
             clusters = tiles;
         }
+    }
+    if (l0) {
+        // slack of a light cluster = one tile's main loop (measured ~0.465 us per K block of the 240-wide tile)
+        const L0Plan plan = l0_plan(clusters, tiles, p.tiles_m, (int)(K / 128), (double)(K / 128) * 0.465 + 0.6,
+                                    ctx->l0_force_splits, ctx->l0_force_fill);
+        p.l0_splits = plan.splits;
+        p.l0_kb_per_split = plan.kb_per_split;
+        p.l0_light0 = plan.light0;
+        p.l0_fill = plan.fill;
+        p.l0_partial = lora->l0_partial;
+        p.l0_tickets = lora->l0_tickets;
+        p.l0_ready = lora->l0_ready;
+        p.l0_epoch = ++ctx->l0_epoch;
+        p.l0_done = lora->l0_ready + L0_WORDS_BYTES / 4;
+        ctx->l0_done_total += (uint32_t)(p.tiles_m * Cfg::CG * 4);
+        p.l0_done_target = ctx->l0_done_total;
+        p.T = static_cast<uint16_t*>(const_cast<void*>(lora->T));
+        p.ldt = lora->ldt;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(clusters * Cfg::CG));
@@ -206,35 +309,41 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     attr[1].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, te, ty, tt, tla, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, te, ty, tt, tla, tx, tlb, p);
     if (e != cudaSuccess) return LYNX_ERR_CUDA;
     ctx->launches++;
     return LYNX_OK;
 }
 
+// Tile configuration for (M, N, K): the development override, else the smallest modelled time.
+// CTA-pair tiles 256 x {256, 240, 192, 128}.  A sparse MMA takes the same time whatever its N
+// (up to 256), so wide tiles win; 240 is the widest that still double-buffers the accumulator.
+// Model: rounds of tiles over the CTA pairs x (K blocks x measured time per K block + exposed
+// epilogue).  Per-K-block times (us) are measured B200 figures for each tile shape; the 256-wide
+// tile has one accumulator buffer, so its epilogue is not hidden.
+int pick_gemm_cfg(const lynx_ctx* ctx, int64_t M, int64_t N, int64_t K, int lora_steps) {
+    if (ctx->gemm_cfg != 0) return ctx->gemm_cfg;
+    const int pairs = ctx->num_sms / 2;
+    const double kb = (double)(K / 128) + lora_steps;
+    struct { int id, bn; double t_kb, epi; } cand[4] = {
+        {7, 240, 0.465, 0.6}, {5, 256, 0.50, 3.0}, {4, 192, 0.415, 0.6}, {6, 128, 0.345, 0.5}};
+    double best = 1e30;
+    int cfg = 7;
+    for (auto& c : cand) {
+        const int64_t tiles = ((M + 255) / 256) * ((N + c.bn - 1) / c.bn);
+        const double rounds = (double)((tiles + pairs - 1) / pairs);
+        const double t = rounds * (kb * c.t_kb + c.epi);
+        if (t < best) { best = t; cfg = c.id; }
+    }
+    return cfg;
+}
+// every tile but the 2-CTA 256 x 128 one has room in its W slot for a phase-0 stage
+bool cfg_supports_l0(int cfg) { return cfg >= 1 && cfg <= 7 && cfg != 6; }
+
 lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K, const void* W,
                         int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp, const LoraArgs* lora, void* Y,
-                        int64_t ldy, cudaStream_t st) {
-    int cfg = ctx->gemm_cfg;
-    if (cfg == 0) {
-        // CTA-pair tiles 256 x {256, 240, 192, 128}.  A sparse MMA takes the same time whatever its N
-        // (up to 256), so wide tiles win; 240 is the widest that still double-buffers the
-        // accumulator.  Pick the tile with the smallest modelled time:
-        // rounds of tiles over the CTA pairs x (K blocks x measured time per K block + exposed
-        // epilogue).  Per-K-block times (us) are measured B200 figures for each tile shape; the
-        // 256-wide tile has one accumulator buffer, so its epilogue is not hidden.
-        const int pairs = ctx->num_sms / 2;
-        const double kb = (double)(K / 128);
-        struct { int id, bn; double t_kb, epi; } cand[4] = {
-            {7, 240, 0.465, 0.6}, {5, 256, 0.50, 3.0}, {4, 192, 0.415, 0.6}, {6, 128, 0.345, 0.5}};
-        double best = 1e30;
-        for (auto& c : cand) {
-            const int64_t tiles = ((M + 255) / 256) * ((N + c.bn - 1) / c.bn);
-            const double rounds = (double)((tiles + pairs - 1) / pairs);
-            const double t = rounds * ((kb + (lora ? lora->R / 64 : 0)) * c.t_kb + c.epi);
-            if (t < best) { best = t; cfg = c.id; }
-        }
-    }
+                        int64_t ldy, cudaStream_t st, int cfg = 0) {
+    if (cfg == 0) cfg = pick_gemm_cfg(ctx, M, N, K, lora ? lora->R / 64 : 0);
 #define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st
     switch (cfg) {
         case 1: return launch_gemm_cfg<GemmCfg<128, 1, 4, 1>>(LYNX_GEMM_ARGS);
@@ -333,8 +442,15 @@ LoraWsLayout lora_ws_layout(int num_sms, int64_t M, int64_t K, int R) {
     lora_split_plan(num_sms, M, K, &splits, &per);
     LoraWsLayout L;
     const size_t tiles_m = (size_t)((M + 127) / 128);
+    size_t partial = splits > 1 ? tiles_m * splits * 128 * (size_t)R * 4 : 0;
+    if (R == 64) {
+        // the in-GEMM down projection: 256-row blocks over CTA pairs, or 128-row blocks over single CTAs
+        // (the same bytes whether the blocks are 256 rows over CTA pairs or 128 rows over single CTAs)
+        const size_t f = (size_t)((M + 255) / 256) * L0_MAX_SPLITS * 256 * 64 * 4;
+        if (f > partial) partial = f;
+    }
     L.partial = 0;
-    size_t off = align_up(splits > 1 ? tiles_m * splits * 128 * (size_t)R * 4 : 0, 1024);
+    size_t off = align_up(partial, 1024);
     L.T = off;
     off = align_up(off + (size_t)M * R * 2, 1024);
     L.total = off;
@@ -426,8 +542,8 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
         return LYNX_ERR_CUDA;
     }
     *ctx->err_host = DEV_OK;
-    if (cudaMalloc(reinterpret_cast<void**>(&ctx->tickets), PRUNE_TICKET_BYTES + LORA_TICKET_BYTES) != cudaSuccess ||
-        cudaMemset(ctx->tickets, 0, PRUNE_TICKET_BYTES + LORA_TICKET_BYTES) != cudaSuccess) {
+    if (cudaMalloc(reinterpret_cast<void**>(&ctx->tickets), TICKET_ALLOC_BYTES) != cudaSuccess ||
+        cudaMemset(ctx->tickets, 0, TICKET_ALLOC_BYTES) != cudaSuccess) {
         cudaFreeHost(ctx->err_host);
         delete ctx;
         return LYNX_ERR_WORKSPACE;
@@ -438,6 +554,12 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
     if (env) ctx->pdl = atoi(env);
     env = getenv("LYNX_STREAMK");  // 1 turns the stream-K tail on
     if (env) ctx->streamk = atoi(env);
+    env = getenv("LYNX_LORA_FUSE");  // 0: down projection of the low-rank branch as its own kernel
+    if (env) ctx->lora_fuse = atoi(env);
+    env = getenv("LYNX_L0_SPLITS");  // development overrides: K splits of the in-GEMM down projection,
+    if (env) ctx->l0_force_splits = atoi(env);
+    env = getenv("LYNX_L0_FILL");  // and items per light cluster (0: round-robin over all clusters)
+    if (env) ctx->l0_force_fill = atoi(env);
     env = getenv("LYNX_PRUNE_TPU");  // development override: 128-element K blocks per warp
     if (env) ctx->prune_tpu = atoi(env);
     *out = ctx;
@@ -602,6 +724,13 @@ lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int6
         return launch_fused(ctx, X, M, K, ldx, W, N, ldw, bias, mode == LYNX_COMP_ROW ? 1 : 0, residual, ldr, Y, ldy,
                             static_cast<cudaStream_t>(stream));
     }
+    // every argument is checked before the first launch
+    if (!X || !W || !Y) return LYNX_ERR_INVALID_ARG;
+    if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    if (ldx < K || ldw < K || ldy < N || (residual && ldr < N)) return LYNX_ERR_INVALID_ARG;
+    if (!aligned16(W) || !aligned16(Y) || (ldw % 8) || (ldy % 8) || (bias && !aligned16(bias)) ||
+        (residual && (!aligned16(residual) || (ldr % 8))))
+        return LYNX_ERR_ALIGNMENT;
     ScratchLayout L = scratch_layout(M, N, K);
     {
         std::lock_guard<std::mutex> lock(ctx->mu);
@@ -707,6 +836,14 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
     if (s != LYNX_OK) return s;
     if ((s = check_lora_rank(R)) != LYNX_OK) return s;
     if (N < 8 || !LA || !LB) return LYNX_ERR_INVALID_ARG;
+    // every argument is checked before the first launch
+    if (!X || !W || !Y) return LYNX_ERR_INVALID_ARG;
+    if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    if (ldx < K || ldw < K || ldy < N || ldla < R || ldlb < K || (residual && ldr < N)) return LYNX_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(LA) || !aligned16(LB) || (ldx % 8) ||
+        (ldw % 8) || (ldy % 8) || (ldla % 8) || (ldlb % 8) || (bias && !aligned16(bias)) ||
+        (residual && (!aligned16(residual) || (ldr % 8))))
+        return LYNX_ERR_ALIGNMENT;
     ScratchLayout L = scratch_layout(M, N, K);
     const LoraWsLayout LL = lora_ws_layout(ctx->num_sms, M, K, (int)R);
     {
@@ -721,12 +858,28 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
     void* T = static_cast<char*>(ctx->lora_ws) + LL.T;
     s = lynx_prune_compress(ctx, X, M, K, ldx, values, meta, scale, mode, stream);
     if (s != LYNX_OK) return s;
-    s = lynx_lora_down(ctx, X, M, K, ldx, LB, R, ldlb, scale, T, R, stream);
-    if (s != LYNX_OK) return s;
     lynx_comp comp;
     comp.row_scale = scale;
     comp.residual = residual;
     comp.ldr = ldr;
+    const int cfg = pick_gemm_cfg(ctx, M, N, K, (int)(R / 64));
+    const bool groups_fit = (size_t)((M + 255) / 256) * 8 * 4 <= L0_WORDS_BYTES;
+    if (ctx->lora_fuse && R == 64 && cfg_supports_l0(cfg) && !ctx->streamk && groups_fit) {
+        // two launches: the GEMM kernel computes T = (X L_B^T) / s itself before its first tile
+        char* ws = static_cast<char*>(ctx->lora_ws);
+        LoraArgs lora{T, R, LA, ldla, (int)R};
+        lora.X = X;
+        lora.ldx = ldx;
+        lora.LB = LB;
+        lora.ldlb = ldlb;
+        lora.l0_partial = reinterpret_cast<float*>(ws + LL.partial);
+        lora.l0_tickets = ctx->tickets + (PRUNE_TICKET_BYTES + LORA_TICKET_BYTES) / 4;
+        lora.l0_ready = lora.l0_tickets + L0_WORDS_BYTES / 4;
+        return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &comp, &lora, Y, ldy,
+                           static_cast<cudaStream_t>(stream), cfg);
+    }
+    s = lynx_lora_down(ctx, X, M, K, ldx, LB, R, ldlb, scale, T, R, stream);
+    if (s != LYNX_OK) return s;
     return lynx_sparse_linear_lora(ctx, values, meta, M, K, W, N, ldw, bias, &comp, T, R, LA, R, ldla, Y, ldy, stream);
 }
 

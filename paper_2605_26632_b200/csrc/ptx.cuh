@@ -95,6 +95,39 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
 __device__ __forceinline__ void st_release_gpu(uint32_t* p, uint32_t v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+// Ticket counter: the add releases this thread's earlier writes (and, by cumulativity, writes of
+// other threads ordered before it by a barrier) and acquires those of the threads that drew
+// earlier tickets -- one fence pair instead of separate __threadfence() calls around a relaxed add.
+__device__ __forceinline__ uint32_t atom_add_acq_rel_gpu(uint32_t* p, uint32_t v) {
+    uint32_t old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+__device__ __forceinline__ void red_add_release_gpu(uint32_t* p, uint32_t v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// Bounded wait until four consecutive words all equal `want` (the four loads of a round are in
+// flight together).  Same limit and abort protocol as flag_wait.
+__device__ __forceinline__ bool flag_wait4(const uint32_t* flags, uint32_t want, volatile uint32_t* cta_abort,
+                                           uint32_t* dev_error) {
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        const uint32_t a = ld_acquire_gpu(flags), b = ld_acquire_gpu(flags + 1), c = ld_acquire_gpu(flags + 2),
+                       d = ld_acquire_gpu(flags + 3);
+        if (a == want && b == want && c == want && d == want) return true;
+        if ((it & 0x3f) == 0x3f) {
+            if (*cta_abort) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) {
+                *cta_abort = 1;
+                atomicExch(dev_error, (uint32_t)DEV_TIMEOUT);
+                __threadfence_system();
+                return false;
+            }
+        }
+    }
+}
 __device__ __forceinline__ bool flag_wait(const uint32_t* flag, uint32_t want, volatile uint32_t* cta_abort,
                                           uint32_t* dev_error) {
     uint64_t t0 = 0;
@@ -169,6 +202,11 @@ __device__ __forceinline__ void tma_store_wait_all() {
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA store source)
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// generic-proxy accesses to global memory ordered against async-proxy (TMA) accesses to it
+__device__ __forceinline__ void fence_proxy_async_global() {
+    asm volatile("fence.proxy.async.global;" ::: "memory");
 }
 
 // Programmatic dependent launch: a kernel launched with the "programmatic stream serialization"

@@ -21,6 +21,17 @@
 // L_A in the W slot, and the issuer adds T L_A^T with four DENSE tcgen05.mma (K = 16 each) into
 // the same accumulator, so Y_r never exists in memory and the epilogue's s_m * acc restores it.
 //
+// With l0_fused the kernel also computes T itself before its first tile ("phase 0"): the work
+// items (256-row block, K split) of X L_B^T are dealt round-robin to the clusters and run through
+// the same ring (a stage then holds two 128 x 64 boxes of the DENSE X and two R-row boxes of L_B,
+// eight dense K = 16 steps) into a 64-column accumulator.  Each epilogue warp writes its 32 rows as
+// an fp32 partial, takes a ticket of its 32-row group, and the warp that draws the group's last
+// ticket adds the splits in ascending order, multiplies by 1 / s_m, writes the bf16 rows of T and
+// publishes the group's ready word (the launch epoch).  The producer waits (bounded) for the
+// four ready words of its rows before it loads a tile's T box -- by then a whole main loop has
+// passed, so the wait is normally already satisfied.  Every cluster finishes its phase-0 items
+// before it can wait for anyone, so the waits cannot deadlock.
+//
 // CG == 2: the pair computes a 256 x BN tile; each CTA stages its own 128 rows of A and
 // metadata and its own BN/2 rows of W (plain TMA loads, no multicast), the leader CTA issues
 // cta_group::2 MMAs, and each CTA drains its own 128 accumulator rows.
@@ -44,6 +55,18 @@ struct GemmParams {
     uint32_t* sk_flags;
     uint32_t sk_epoch;
     int lora_steps;  // R / 64 extra dense stages per tile (0 = no low-rank branch)
+    // phase 0 (l0_fused): T = (X L_B^T) / s computed by this launch, R = 64
+    int l0_fused;
+    int l0_splits, l0_kb_per_split;  // K splits per 256-row block, 128-element K blocks per split
+    int l0_light0, l0_fill;          // see L0Schedule
+    float* l0_partial;     // [row block][split][16 pieces][rows of the block] float4
+    uint32_t* l0_tickets;  // one word per 32-row group, zero between launches
+    uint32_t* l0_ready;    // one word per 32-row group: epoch of the launch that finished its T rows
+    uint32_t l0_epoch;
+    uint32_t* l0_done;     // running count of published groups over all launches of the context
+    uint32_t l0_done_target;  // its value once this launch has published all of its groups
+    uint16_t* T;           // [M x 64] bf16, leading dimension ldt
+    int64_t ldt;
 };
 
 // Work distribution over C persistent clusters.  The first floor(T/C)*C tiles go round-robin,
@@ -110,6 +133,31 @@ struct TileSchedule {
     }
 };
 
+// Which cluster runs which phase-0 item.  With T tiles over C clusters the clusters c >= T % C
+// ("light") have one tile fewer than the others, i.e. a whole tile time of slack: the first
+// light * fill items go to them, round-robin (the host sets fill so that either all items fit
+// there or fill = 0), the rest round-robin over all clusters.  light0 = C: no light clusters.
+struct L0Schedule {
+    int items, C, light0, L, cap;
+    __device__ L0Schedule(int items_, int clusters, int light0_, int fill) : items(items_), C(clusters), light0(light0_) {
+        L = C - light0;
+        cap = L * fill;
+        if (cap > items) cap = items;
+    }
+    __device__ int light_count(int c) const {
+        const int lc = c - light0;
+        return (lc >= 0 && cap > lc) ? (cap - lc + L - 1) / L : 0;
+    }
+    __device__ int count(int c) const {
+        const int rest = items - cap;
+        return light_count(c) + ((rest > c) ? (rest - c + C - 1) / C : 0);
+    }
+    __device__ int item(int c, int li) const {
+        const int nl = light_count(c);
+        return (li < nl) ? (c - light0) + li * L : cap + c + (li - nl) * C;
+    }
+};
+
 template <int BN_, int CG_, int STAGES_, int CBUFS_>
 struct GemmCfg {
     static constexpr int BN = BN_, CG = CG_, STAGES = STAGES_, CBUFS = CBUFS_;
@@ -139,6 +187,12 @@ struct GemmCfg {
     static_assert(B_HALF_BYTES % 1024 == 0, "swizzle atoms need 1024-byte aligned tiles");
     static_assert(E_COL0 % 4 == 0 && E_COL0 + 4 * STAGES <= TMEM_COLS, "tensor memory budget");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+    // phase 0 stage (rank 64): L_B boxes at the start of the W slot, second X box behind them
+    static constexpr int L0_R = 64;
+    static constexpr int L0_LB_BYTES = (L0_R / CG) * 64 * 2;
+    static constexpr int L0_X2_OFF = (2 * L0_LB_BYTES + 1023) / 1024 * 1024;
+    static constexpr int L0_STAGE_BYTES = 2 * A_BYTES + 2 * L0_LB_BYTES;
+    static constexpr bool L0_OK = L0_X2_OFF + A_BYTES <= B_BYTES;
 };
 
 // Instruction descriptor of tcgen05.mma.sp kind::f16: bf16 x bf16 -> fp32, both operands
@@ -157,6 +211,7 @@ __global__ void __launch_bounds__(Cfg::THREADS, 1)
 sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                    const __grid_constant__ CUtensorMap tmap_e, const __grid_constant__ CUtensorMap tmap_y,
                    const __grid_constant__ CUtensorMap tmap_t, const __grid_constant__ CUtensorMap tmap_la,
+                   const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_lb,
                    const GemmParams p) {
     constexpr int CG = Cfg::CG, STAGES = Cfg::STAGES, BN = Cfg::BN;
     extern __shared__ uint8_t smem_raw[];
@@ -181,6 +236,10 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     const int kblocks = (int)(p.K / Cfg::BK);
     const TileSchedule sched(num_tiles, num_clusters, kblocks, p.sk_partial != nullptr);
     const int num_items = sched.count(cluster_id);
+    // phase 0 items of this cluster: item -> (row block = item % tiles_m, K split = item / tiles_m)
+    const int l0_items = (Cfg::L0_OK && p.l0_fused) ? p.tiles_m * p.l0_splits : 0;
+    const L0Schedule l0s(l0_items, num_clusters, p.l0_light0, p.l0_fill);
+    const int n0 = l0s.count(cluster_id);
 
     if (threadIdx.x == 0) {
         *cta_abort = 0;
@@ -201,6 +260,10 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             prefetch_tmap(&tmap_t);
             prefetch_tmap(&tmap_la);
         }
+        if (p.l0_fused) {
+            prefetch_tmap(&tmap_x);
+            prefetch_tmap(&tmap_lb);
+        }
     }
     if (warp == 1) {
         tmem_alloc<CG>(smem_u32(tmem_slot), Cfg::TMEM_COLS);
@@ -220,7 +283,44 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             uint32_t stage = 0, phase = 0;
             uint32_t issued = 0;
             bool ok = true;
+            bool l0_all_done = false;
             const uint32_t full0 = (CG == 2) ? mapa(bar_full, 0) : bar_full;  // leader's barriers
+            if constexpr (Cfg::L0_OK) {
+                // phase 0: dense X boxes and L_B boxes of this cluster's (row block, K split) items
+                for (int li = 0; li < n0 && ok; ++li) {
+                    const int item = l0s.item(cluster_id, li);
+                    const int tmb = item % p.tiles_m, split = item / p.tiles_m;
+                    const int m0 = (tmb * CG + (int)rank) * Cfg::BM;
+                    const int lb_row0 = (int)rank * (Cfg::L0_R / CG);
+                    const int k0 = split * p.l0_kb_per_split;
+                    const int k1 = (k0 + p.l0_kb_per_split < kblocks) ? k0 + p.l0_kb_per_split : kblocks;
+                    for (int kb = k0; kb < k1; ++kb) {
+                        if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, cta_abort, p.dev_error)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t a_dst = sA + stage * Cfg::A_BYTES;
+                        const uint32_t b_dst = sB + stage * Cfg::B_BYTES;
+                        if constexpr (CG == 1) {
+                            const uint32_t bar = bar_full + 8 * stage;
+                            mbar_arrive_expect_tx(bar, Cfg::L0_STAGE_BYTES);
+                            tma_load_2d(a_dst, &tmap_x, kb * 128, m0, bar);
+                            tma_load_2d(b_dst + Cfg::L0_X2_OFF, &tmap_x, kb * 128 + 64, m0, bar);
+                            tma_load_2d(b_dst, &tmap_lb, kb * 128, lb_row0, bar);
+                            tma_load_2d(b_dst + Cfg::L0_LB_BYTES, &tmap_lb, kb * 128 + 64, lb_row0, bar);
+                        } else {
+                            const uint32_t bar = full0 + 8 * stage;
+                            if (leader) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * Cfg::L0_STAGE_BYTES);
+                            tma_load_2d_pair(a_dst, &tmap_x, kb * 128, m0, bar);
+                            tma_load_2d_pair(b_dst + Cfg::L0_X2_OFF, &tmap_x, kb * 128 + 64, m0, bar);
+                            tma_load_2d_pair(b_dst, &tmap_lb, kb * 128, lb_row0, bar);
+                            tma_load_2d_pair(b_dst + Cfg::L0_LB_BYTES, &tmap_lb, kb * 128 + 64, lb_row0, bar);
+                        }
+                        ++issued;
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    }
+                }
+            }
             for (int wi = 0; wi < num_items && ok; ++wi) {
                 const WorkItem w = sched.get(cluster_id, wi);
                 const int tm = w.tile % p.tiles_m, tn = w.tile / p.tiles_m;
@@ -262,6 +362,15 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                             ok = false;
                             break;
                         }
+                        if (l0_items > 0 && j == 0 && !l0_all_done) {
+                            // T rows of this CTA's 128 rows come from phase 0 of this launch: one look at
+                            // the count of published groups (once complete, no tile looks again), else
+                            // wait for the four ready words of these rows
+                            if (ld_acquire_gpu(p.l0_done) == p.l0_done_target) l0_all_done = true;
+                            else ok = flag_wait4(p.l0_ready + (tm * CG + (int)rank) * 4, p.l0_epoch, cta_abort, p.dev_error);
+                            if (!ok) break;
+                            fence_proxy_async_global();
+                        }
                         constexpr uint32_t LORA_BYTES = Cfg::A_BYTES + Cfg::B_HALF_BYTES;
                         const uint32_t a_dst = sA + stage * Cfg::A_BYTES;
                         const uint32_t b_dst = sB + stage * Cfg::B_BYTES;
@@ -295,11 +404,56 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             constexpr uint32_t BH = Cfg::B_HALF_BYTES >> 4;
             uint32_t stage = 0, phase = 0;
             bool ok = true;
+            if constexpr (Cfg::L0_OK) {
+                // phase 0: eight dense K = 16 steps per stage into the first 64 accumulator columns
+                constexpr uint32_t idesc_l0 = make_idesc_sp_bf16(Cfg::BM * CG, Cfg::L0_R) & ~(1u << 2);
+                for (int li = 0; li < n0 && ok; ++li) {
+                    const int item = l0s.item(cluster_id, li);
+                    const int split = item / p.tiles_m;
+                    const int k0 = split * p.l0_kb_per_split;
+                    const int k1 = (k0 + p.l0_kb_per_split < kblocks) ? k0 + p.l0_kb_per_split : kblocks;
+                    const int acc = (Cfg::ACC_STAGES == 2) ? (li & 1) : 0;
+                    const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((li >> 1) & 1) : (li & 1);
+                    if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, cta_abort, p.dev_error)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * BN;
+                    uint32_t accumulate = 0;
+                    for (int kb = k0; kb < k1; ++kb) {
+                        if (!mbar_wait(bar_full + 8 * stage, phase, cta_abort, p.dev_error)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t a_lo = a_lo0 + stage * (Cfg::A_BYTES >> 4);
+                        const uint32_t b_lo = b_lo0 + stage * (Cfg::B_BYTES >> 4);
+                        const uint32_t a2_lo = b_lo + (Cfg::L0_X2_OFF >> 4);
+                        const uint32_t b2_lo = b_lo + (Cfg::L0_LB_BYTES >> 4);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            mma_bf16_lh<CG>(d_tmem, a_lo + 2 * i, b_lo + 2 * i, desc_hi, idesc_l0, accumulate);
+                            accumulate = 1u;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            mma_bf16_lh<CG>(d_tmem, a2_lo + 2 * i, b2_lo + 2 * i, desc_hi, idesc_l0, 1u);
+                        if constexpr (CG == 1) tc_commit(bar_empty + 8 * stage);
+                        else tc_commit_pair(bar_empty + 8 * stage, 0x3);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    }
+                    if (!ok) break;
+                    if constexpr (CG == 1) tc_commit(bar_tfull + 8 * acc);
+                    else tc_commit_pair(bar_tfull + 8 * acc, 0x3);
+                }
+            }
             int it = 0;
             for (; it < num_items && ok; ++it) {
                 const WorkItem w = sched.get(cluster_id, it);
-                const int acc = (Cfg::ACC_STAGES == 2) ? (it & 1) : 0;
-                const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((it >> 1) & 1) : (it & 1);
+                const int gi = n0 + it;  // accumulator buffers alternate over phase 0 items and tiles alike
+                const int acc = (Cfg::ACC_STAGES == 2) ? (gi & 1) : 0;
+                const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((gi >> 1) & 1) : (gi & 1);
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, cta_abort, p.dev_error)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
@@ -358,11 +512,114 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         const uint32_t tempty0 = (CG == 2) ? mapa(bar_tempty, 0) : bar_tempty;
         int it = 0, cb = 0;
         bool alive = true;
+        if constexpr (Cfg::L0_OK) {
+            // ---- phase 0: drain the 64-column accumulator of each (row block, K split) item ----
+            constexpr int PIECES = Cfg::L0_R / 4;  // float4 pieces per row
+            constexpr int BLOCK_ROWS = Cfg::BM * CG;
+            for (int li = 0; li < n0 && alive; ++li) {
+                const int item = l0s.item(cluster_id, li);
+                const int tmb = item % p.tiles_m, split = item / p.tiles_m;
+                const int acc = (Cfg::ACC_STAGES == 2) ? (li & 1) : 0;
+                const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((li >> 1) & 1) : (li & 1);
+                const int row_in_block = (int)rank * Cfg::BM + q * 32 + lane;
+                const int64_t row = (int64_t)tmb * BLOCK_ROWS + row_in_block;
+                // the row's scale is fetched while the item's K loop runs (a global load costs over a
+                // microsecond once the main loops saturate the memory system); T = acc * (1 / s)
+                float inv_s = 1.0f;
+                if (p.row_scale != nullptr && row < p.M) {
+                    const float sc = __ldg(p.row_scale + row);
+                    inv_s = (sc == 0.0f) ? 0.0f : __frcp_rn(sc);
+                }
+                if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, cta_abort, p.dev_error)) {
+                    alive = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+                uint32_t v[64];
+                tmem_ld_32x32b_x32(t_row, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                tmem_ld_32x32b_x32(t_row + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if constexpr (CG == 1) mbar_arrive(bar_tempty + 8 * acc);
+                    else mbar_arrive_cluster(tempty0 + 8 * acc);
+                }
+                const int group = (tmb * CG + (int)rank) * 4 + q;  // this warp's 32 rows
+                bool last = true;
+                if (p.l0_splits > 1) {
+                    // partial: [row block][split][piece][row] float4 -> a warp's piece is 512 contiguous bytes
+                    float4* dst = reinterpret_cast<float4*>(p.l0_partial) +
+                                  ((size_t)tmb * p.l0_splits + split) * PIECES * BLOCK_ROWS + row_in_block;
+#pragma unroll
+                    for (int j = 0; j < PIECES; ++j)
+                        __stcg(dst + (size_t)j * BLOCK_ROWS,
+                               make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                           __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+                    // the warp's partial rows are ordered before lane 0's releasing add by the warp barrier;
+                    // the add also acquires the partials of the warps that drew the earlier tickets
+                    __syncwarp();
+                    uint32_t ticket = 0;
+                    if (lane == 0) ticket = atom_add_acq_rel_gpu(p.l0_tickets + group, 1u);
+                    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+                    __syncwarp();  // lane 0's acquire ordered before every lane's loads of the partials
+                    last = ticket == (uint32_t)p.l0_splits - 1;
+                    if (last) {
+                        // ascending split order whichever warp is last: reproducible bit for bit
+                        const float4* src = reinterpret_cast<const float4*>(p.l0_partial) +
+                                            (size_t)tmb * p.l0_splits * PIECES * BLOCK_ROWS + row_in_block;
+#pragma unroll
+                        for (int j = 0; j < 64; ++j) v[j] = 0u;  // +0.0f
+                        // one batch of 16 independent loads per split: every batch costs a full L2 round
+                        // trip under the main loop's traffic, so few large batches
+                        for (int sp = 0; sp < p.l0_splits; ++sp) {
+                            float4 pa[PIECES];
+#pragma unroll
+                            for (int j = 0; j < PIECES; ++j)
+                                pa[j] = __ldcg(src + ((size_t)sp * PIECES + j) * BLOCK_ROWS);
+#pragma unroll
+                            for (int j = 0; j < PIECES; ++j) {
+                                v[4 * j] = __float_as_uint(__uint_as_float(v[4 * j]) + pa[j].x);
+                                v[4 * j + 1] = __float_as_uint(__uint_as_float(v[4 * j + 1]) + pa[j].y);
+                                v[4 * j + 2] = __float_as_uint(__uint_as_float(v[4 * j + 2]) + pa[j].z);
+                                v[4 * j + 3] = __float_as_uint(__uint_as_float(v[4 * j + 3]) + pa[j].w);
+                            }
+                        }
+                    }
+                }
+                if (last) {
+                    if (row < p.M) {
+                        uint4* dst = reinterpret_cast<uint4*>(p.T + row * p.ldt);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float a0 = __uint_as_float(v[8 * j + 2 * e]), a1 = __uint_as_float(v[8 * j + 2 * e + 1]);
+                                o[e] = pack_bf16x2(a0 * inv_s, a1 * inv_s);
+                            }
+                            dst[j] = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                    // T rows written with generic stores are read by TMA: order both proxies, then publish
+                    // (the releasing store orders every lane's rows, which the warp barrier put before it)
+                    fence_proxy_async_global();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (p.l0_splits > 1) p.l0_tickets[group] = 0;  // ready for the next launch
+                        st_release_gpu(p.l0_ready + group, p.l0_epoch);
+                        red_add_release_gpu(p.l0_done, 1u);
+                    }
+                }
+            }
+        }
         for (; it < num_items && alive; ++it) {
             const WorkItem w = sched.get(cluster_id, it);
             const int tm = w.tile % p.tiles_m, tn = w.tile / p.tiles_m;
-            const int acc = (Cfg::ACC_STAGES == 2) ? (it & 1) : 0;
-            const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((it >> 1) & 1) : (it & 1);
+            const int gi = n0 + it;
+            const int acc = (Cfg::ACC_STAGES == 2) ? (gi & 1) : 0;
+            const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((gi >> 1) & 1) : (gi & 1);
             if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, cta_abort, p.dev_error)) break;
             tc_fence_after();
             const int m0 = (tm * CG + (int)rank) * Cfg::BM + q * 32;
@@ -483,8 +740,8 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 cb = (cb + 1 == Cfg::CBUFS) ? 0 : cb + 1;
             }
             if (w.kind == 1) {
-                // publish: all lanes' stores, then the ready word of this (slot, warp)
-                __threadfence();
+                // publish: all lanes' stores (ordered before lane 0 by the warp barrier), then the
+                // releasing store of the ready word of this (slot, warp)
                 __syncwarp();
                 if (lane == 0) st_release_gpu(p.sk_flags + cluster_id * 8 + my_flag, p.sk_epoch);
             }
