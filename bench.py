@@ -50,6 +50,7 @@ def parse_args():
     ap.add_argument("--comp", default="row", choices=["none", "row", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-lora", action="store_true", help="skip the extra measurement of the layer with the low-rank branch")
     return ap.parse_args()
 
 
@@ -333,6 +334,30 @@ def main():
     dense_ms = d0.elapsed_time(d1) / args.steps
     t_wall2 = time.time()
 
+    # the same layer with the rank-64 low-rank branch (Y = Y_s + X (L_A L_B)^T), outside the headline
+    # number: its cost on top of the step, same rotation and event timing
+    lora = None
+    if not args.no_lora:
+        R = 64
+        LA, LB = inputs.make_lora(N, K, R, wl.seed)
+        LA, LB = LA.cuda(), LB.cuda()
+        lx.reserve_lora(M, K, R)
+        for i in range(3):
+            lx.act_sparse_linear_lora(Xs[i % NSETS], Ws[i % NSETS], LA, LB, bias, comp_mode, None, Ys[i % NSETS])
+        torch.cuda.synchronize()
+        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0.record(stream)
+        for i in range(args.steps):
+            j = i % NSETS
+            lx.act_sparse_linear_lora(Xs[j], Ws[j], LA, LB, bias, comp_mode, None, Ys[j])
+        l1.record(stream)
+        torch.cuda.synchronize()
+        lora_ms = l0.elapsed_time(l1) / args.steps
+        lora = {"rank": R, "ms_per_step": lora_ms, "overhead_vs_step": lora_ms / (total_ms / args.steps) - 1.0,
+                "speedup_vs_dense_bf16_without_lora": dense_ms / lora_ms,
+                "how": "lynx_act_sparse_linear_lora: prune/compress + sparse GEMM whose launch also computes "
+                       "T = (X L_B^T) / s and adds T L_A^T in its accumulator"}
+
     # end to end through the host-buffer entry point: pinned X in, pinned Y out, every step
     e2e = None
     if not args.no_e2e:
@@ -401,6 +426,7 @@ def main():
                            "peak_kind": f"hbm_gbs ({peaks['source']})"},
         "clocks": clocks,
         "e2e": e2e,
+        "lora": lora,
         "gpu_launches": int(launches),
     }
 

@@ -204,8 +204,14 @@ LYNX_API lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_ho
  *   order in which CTAs finish.
  * lynx_sparse_linear_lora:  lynx_sparse_linear plus the T L_A^T term; T must come from
  *   lynx_lora_down called with the same row_scale that comp carries.
- * lynx_act_sparse_linear_lora:  the whole layer: prune/compress, down projection, sparse GEMM
- *   with the low-rank steps, back to back on `stream`, intermediates in the context's scratch.
+ * lynx_act_sparse_linear_lora:  the whole layer, intermediates in the context's scratch.  For
+ *   R = 64 it is two launches: prune/compress, then a sparse GEMM launch that first computes T
+ *   itself (its clusters share the (row block, K split) items of X L_B^T, publish the T rows
+ *   through ready words, and wait -- bounded -- for the rows a tile needs) and then runs the
+ *   tiles with the low-rank steps.  Otherwise (R = 128) three launches: prune/compress,
+ *   lynx_lora_down, lynx_sparse_linear_lora.  Both give Y within the stated tolerance of the
+ *   definition; they may differ from each other in the last bit of T (different K splits, and
+ *   the in-launch form multiplies by 1/s_m where lynx_lora_down divides).
  * Pointers and leading dimensions follow the 16-byte rule of the other entry points.
  */
 LYNX_API lynx_status lynx_reserve_lora(lynx_ctx* ctx, int64_t M, int64_t K, int64_t R);

@@ -246,12 +246,12 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     p.T = nullptr;
     p.ldt = 0;
 
-    auto kern = sparse_gemm_kernel<Cfg>;
-    static bool attr_set = false;  // per instantiation
-    if (!attr_set) {
+    auto kern = lora ? sparse_gemm_kernel<Cfg, true> : sparse_gemm_kernel<Cfg, false>;
+    static bool attr_set[2] = {false, false};  // per instantiation
+    if (!attr_set[lora ? 1 : 0]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
             return LYNX_ERR_CUDA;
-        attr_set = true;
+        attr_set[lora ? 1 : 0] = true;
     }
     const int tiles = p.tiles_m * p.tiles_n;
     int clusters = ctx->num_sms / Cfg::CG;

@@ -206,7 +206,9 @@ __host__ __device__ constexpr uint32_t make_idesc_sp_bf16(int m, int n) {
            | ((uint32_t)(m >> 4) << 24);    // M / 16
 }
 
-template <class Cfg>
+// LORA = false is the plain layer: the low-rank stages and phase 0 are compiled out, so the hot
+// kernel carries none of their registers or parameters' uses.
+template <class Cfg, bool LORA>
 __global__ void __launch_bounds__(Cfg::THREADS, 1)
 sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                    const __grid_constant__ CUtensorMap tmap_e, const __grid_constant__ CUtensorMap tmap_y,
@@ -214,6 +216,8 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                    const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_lb,
                    const GemmParams p) {
     constexpr int CG = Cfg::CG, STAGES = Cfg::STAGES, BN = Cfg::BN;
+    constexpr bool L0 = LORA && Cfg::L0_OK;
+    const int lora_steps = LORA ? p.lora_steps : 0;
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment for the swizzled tiles
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -237,9 +241,9 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     const TileSchedule sched(num_tiles, num_clusters, kblocks, p.sk_partial != nullptr);
     const int num_items = sched.count(cluster_id);
     // phase 0 items of this cluster: item -> (row block = item % tiles_m, K split = item / tiles_m)
-    const int l0_items = (Cfg::L0_OK && p.l0_fused) ? p.tiles_m * p.l0_splits : 0;
+    const int l0_items = (L0 && p.l0_fused) ? p.tiles_m * p.l0_splits : 0;
     const L0Schedule l0s(l0_items, num_clusters, p.l0_light0, p.l0_fill);
-    const int n0 = l0s.count(cluster_id);
+    const int l0_n = L0 ? l0s.count(cluster_id) : 0;
 
     if (threadIdx.x == 0) {
         *cta_abort = 0;
@@ -256,11 +260,11 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         prefetch_tmap(&tmap_b);
         prefetch_tmap(&tmap_e);
         prefetch_tmap(&tmap_y);
-        if (p.lora_steps) {
+        if (lora_steps) {
             prefetch_tmap(&tmap_t);
             prefetch_tmap(&tmap_la);
         }
-        if (p.l0_fused) {
+        if (L0 && p.l0_fused) {
             prefetch_tmap(&tmap_x);
             prefetch_tmap(&tmap_lb);
         }
@@ -285,9 +289,9 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             bool ok = true;
             bool l0_all_done = false;
             const uint32_t full0 = (CG == 2) ? mapa(bar_full, 0) : bar_full;  // leader's barriers
-            if constexpr (Cfg::L0_OK) {
+            if constexpr (L0) {
                 // phase 0: dense X boxes and L_B boxes of this cluster's (row block, K split) items
-                for (int li = 0; li < n0 && ok; ++li) {
+                for (int li = 0; li < l0_n && ok; ++li) {
                     const int item = l0s.item(cluster_id, li);
                     const int tmb = item % p.tiles_m, split = item / p.tiles_m;
                     const int m0 = (tmb * CG + (int)rank) * Cfg::BM;
@@ -357,7 +361,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 }
                 // low-rank stages: T box in the A slot, L_A box in the first half of the W slot
                 if (w.kb1 == kblocks) {
-                    for (int j = 0; j < p.lora_steps && ok; ++j) {
+                    for (int j = 0; j < lora_steps && ok; ++j) {
                         if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, cta_abort, p.dev_error)) {
                             ok = false;
                             break;
@@ -404,10 +408,10 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             constexpr uint32_t BH = Cfg::B_HALF_BYTES >> 4;
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            if constexpr (Cfg::L0_OK) {
+            if constexpr (L0) {
                 // phase 0: eight dense K = 16 steps per stage into the first 64 accumulator columns
                 constexpr uint32_t idesc_l0 = make_idesc_sp_bf16(Cfg::BM * CG, Cfg::L0_R) & ~(1u << 2);
-                for (int li = 0; li < n0 && ok; ++li) {
+                for (int li = 0; li < l0_n && ok; ++li) {
                     const int item = l0s.item(cluster_id, li);
                     const int split = item / p.tiles_m;
                     const int k0 = split * p.l0_kb_per_split;
@@ -451,7 +455,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             int it = 0;
             for (; it < num_items && ok; ++it) {
                 const WorkItem w = sched.get(cluster_id, it);
-                const int gi = n0 + it;  // accumulator buffers alternate over phase 0 items and tiles alike
+                const int gi = l0_n + it;  // accumulator buffers alternate over phase 0 items and tiles alike
                 const int acc = (Cfg::ACC_STAGES == 2) ? (gi & 1) : 0;
                 const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((gi >> 1) & 1) : (gi & 1);
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, cta_abort, p.dev_error)) break;
@@ -481,7 +485,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 }
                 if (ok && w.kb1 == kblocks) {
                     constexpr uint32_t idesc_dense = idesc0 & ~(1u << 2);
-                    for (int j = 0; j < p.lora_steps; ++j) {
+                    for (int j = 0; j < lora_steps; ++j) {
                         if (!mbar_wait(bar_full + 8 * stage, phase, cta_abort, p.dev_error)) {
                             ok = false;
                             break;
@@ -512,11 +516,11 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         const uint32_t tempty0 = (CG == 2) ? mapa(bar_tempty, 0) : bar_tempty;
         int it = 0, cb = 0;
         bool alive = true;
-        if constexpr (Cfg::L0_OK) {
+        if constexpr (L0) {
             // ---- phase 0: drain the 64-column accumulator of each (row block, K split) item ----
             constexpr int PIECES = Cfg::L0_R / 4;  // float4 pieces per row
             constexpr int BLOCK_ROWS = Cfg::BM * CG;
-            for (int li = 0; li < n0 && alive; ++li) {
+            for (int li = 0; li < l0_n && alive; ++li) {
                 const int item = l0s.item(cluster_id, li);
                 const int tmb = item % p.tiles_m, split = item / p.tiles_m;
                 const int acc = (Cfg::ACC_STAGES == 2) ? (li & 1) : 0;
@@ -617,7 +621,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         for (; it < num_items && alive; ++it) {
             const WorkItem w = sched.get(cluster_id, it);
             const int tm = w.tile % p.tiles_m, tn = w.tile / p.tiles_m;
-            const int gi = n0 + it;
+            const int gi = l0_n + it;
             const int acc = (Cfg::ACC_STAGES == 2) ? (gi & 1) : 0;
             const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((gi >> 1) & 1) : (gi & 1);
             if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, cta_abort, p.dev_error)) break;

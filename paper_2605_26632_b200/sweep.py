@@ -22,13 +22,20 @@ USE_GRAPH = True
 
 
 def timeloop(fn, nsets, iters, warm=5):
-    """Average device time of one call of fn (ms).  The `iters` calls are captured into one CUDA
-    graph and the graph is replayed, so that launches shorter than the host's per-call cost
-    (tensor-map encoding + launch, ~10 us from Python) are timed at the GPU's pace, not the host's."""
+    """Average device time of one call of fn (ms).  The calls are captured into one CUDA graph and
+    the graph is replayed, so that launches shorter than the host's per-call cost (tensor-map
+    encoding + launch, ~10 us from Python) are timed at the GPU's pace, not the host's.  The
+    number of calls is cut so that one replay lasts about 6 ms: seconds of back-to-back tensor-core
+    work run into the power cap and would time the sustained clocks, not the kernel."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
     for i in range(warm):
         fn(i % nsets)
+    b.record()
     torch.cuda.synchronize()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    est_ms = a.elapsed_time(b) / warm
+    iters = max(4, min(iters, int(6.0 / max(est_ms, 1e-3))))
     if not USE_GRAPH:
         a.record()
         for i in range(iters):
@@ -40,15 +47,17 @@ def timeloop(fn, nsets, iters, warm=5):
     with torch.cuda.graph(g):
         for i in range(iters):
             fn(i % nsets)
-    g.replay()
     torch.cuda.synchronize()
-    reps = 3
-    a.record()
-    for _ in range(reps):
+    best = None
+    for _ in range(3):  # three separate replays with an idle gap; the median is reported
+        torch.cuda.synchronize()
+        a.record()
         g.replay()
-    b.record()
-    torch.cuda.synchronize()
-    return a.elapsed_time(b) / (iters * reps)
+        b.record()
+        torch.cuda.synchronize()
+        t = a.elapsed_time(b) / iters
+        best = [t] if best is None else best + [t]
+    return sorted(best)[1]
 
 
 def main():
