@@ -168,7 +168,11 @@ LYNX_API lynx_status lynx_sparse_linear(lynx_ctx* ctx, const void* values, const
  * Y = act_sparse_linear(X, W, bias, residual) = steps 1-6 above.  SEPARATE runs the two kernels
  * back to back on `stream` with the compressed operands in the context's scratch (grown on
  * demand: see lynx_reserve); FUSED prunes inside the GEMM kernel.  Both give the same values,
- * metadata and (up to fp32 summation order) the same Y.
+ * metadata and (up to fp32 summation order) the same Y.  In SEPARATE + LYNX_COMP_ROW the prune
+ * launch leaves the per-K-split row sums in the scratch and the GEMM's epilogue forms s_m from
+ * them, adding in the order lynx_prune_compress itself uses: Y is bit-identical to calling
+ * lynx_prune_compress and lynx_sparse_linear one after the other, without the scale hand-over
+ * inside the first kernel.
  */
 LYNX_API lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
                                             int64_t ldx, const void* W, int64_t N, int64_t ldw,

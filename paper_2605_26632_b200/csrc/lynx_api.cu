@@ -30,6 +30,7 @@ struct lynx_ctx {
     uint32_t l0_epoch = 0;        // launch counter of the fused down projection (ready words hold it)
     uint32_t l0_done_total = 0;   // groups published by all such launches so far (mod 2^32)
     int l0_force_splits = 0, l0_force_fill = -1;  // development overrides of the phase-0 plan
+    int defer_scale = 1;  // layer calls: row scale summed in the GEMM epilogue (LYNX_DEFER_SCALE=0: in the prune kernel)
     int lora_fuse = 1;            // down projection inside the GEMM launch when the tile allows (LYNX_LORA_FUSE=0: own kernel)
     float* sk_partial = nullptr;  // stream-K partial tiles (one slot per cluster) + ready words
     uint32_t* sk_flags = nullptr;
@@ -94,6 +95,12 @@ constexpr size_t LORA_TICKET_BYTES = 64u << 10;  // after the prune tickets: 163
 // at a fixed place of the zero-initialised ticket allocation, whatever shapes the context serves
 constexpr size_t L0_WORDS_BYTES = 256u << 10;
 constexpr size_t TICKET_ALLOC_BYTES = PRUNE_TICKET_BYTES + LORA_TICKET_BYTES + 2 * L0_WORDS_BYTES + 256;  // + done counter
+
+// Row sums a deferred prune launch left in the context's scratch for the GEMM that follows it.
+struct ScaleSrc {
+    const float* partial = nullptr;
+    int ks = 0;
+};
 
 // Low-rank branch operands of the GEMM: T = (X L_B^T) / s [M x R] bf16 and L_A [N x R] bf16.
 struct LoraArgs {
@@ -184,7 +191,7 @@ ScratchLayout scratch_layout(int64_t M, int64_t N, int64_t K) {
 template <class Cfg>
 lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
                             const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
-                            const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st) {
+                            const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st, const ScaleSrc* ss) {
     CUtensorMap ta, tb, te, ty, tt, tla, tx, tlb;
     const uint64_t rb = (uint64_t)((M + 127) / 128), kblocks = (uint64_t)(K / 128);
     if (!make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, values, (uint64_t)M, (uint64_t)(K / 2),
@@ -223,6 +230,8 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     p.lora_steps = lora ? lora->R / 64 : 0;
     p.M = M; p.N = N; p.K = K;
     p.row_scale = comp ? comp->row_scale : nullptr;
+    p.scale_partial = ss ? ss->partial : nullptr;
+    p.scale_ks = ss ? ss->ks : 0;
     p.bias = static_cast<const uint16_t*>(bias);
     p.residual = comp ? static_cast<const uint16_t*>(comp->residual) : nullptr;
     p.ldr = comp ? comp->ldr : 0;
@@ -342,9 +351,9 @@ bool cfg_supports_l0(int cfg) { return cfg >= 1 && cfg <= 7 && cfg != 6; }
 
 lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K, const void* W,
                         int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp, const LoraArgs* lora, void* Y,
-                        int64_t ldy, cudaStream_t st, int cfg = 0) {
+                        int64_t ldy, cudaStream_t st, int cfg = 0, const ScaleSrc* ss = nullptr) {
     if (cfg == 0) cfg = pick_gemm_cfg(ctx, M, N, K, lora ? lora->R / 64 : 0);
-#define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st
+#define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss
     switch (cfg) {
         case 1: return launch_gemm_cfg<GemmCfg<128, 1, 4, 1>>(LYNX_GEMM_ARGS);
         case 2: return launch_gemm_cfg<GemmCfg<192, 1, 3, 1>>(LYNX_GEMM_ARGS);
@@ -560,6 +569,8 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
     if (env) ctx->l0_force_splits = atoi(env);
     env = getenv("LYNX_L0_FILL");  // and items per light cluster (0: round-robin over all clusters)
     if (env) ctx->l0_force_fill = atoi(env);
+    env = getenv("LYNX_DEFER_SCALE");
+    if (env) ctx->defer_scale = atoi(env);
     env = getenv("LYNX_PRUNE_TPU");  // development override: 128-element K blocks per warp
     if (env) ctx->prune_tpu = atoi(env);
     *out = ctx;
@@ -611,13 +622,18 @@ lynx_status lynx_reserve(lynx_ctx* ctx, int64_t M, int64_t N, int64_t K) {
 
 int64_t lynx_launch_count(lynx_ctx* ctx) { return ctx ? ctx->launches : -1; }
 
-lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, void* values,
-                                void* meta, float* row_scale, lynx_comp_mode mode, void* stream) {
+// The prune/compress launch.  defer (ROW mode only): the kernel stops at the per-K-split row sums
+// and `src` tells the following GEMM where they are; its epilogue adds them in the same order the
+// in-kernel finalize would (same bits), which saves the ticket hand-over inside this kernel.
+static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, void* values,
+                              void* meta, float* row_scale, lynx_comp_mode mode, void* stream, bool defer,
+                              ScaleSrc* src) {
     lynx_status s = check_common(ctx, M, K);
     if (s != LYNX_OK) return s;
     if (!X || !values || !meta) return LYNX_ERR_INVALID_ARG;
     if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW && mode != LYNX_COMP_TENSOR) return LYNX_ERR_INVALID_ARG;
-    if (mode != LYNX_COMP_NONE && !row_scale) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_ROW) defer = false;
+    if (mode != LYNX_COMP_NONE && !row_scale && !defer) return LYNX_ERR_INVALID_ARG;
     if (ldx < K) return LYNX_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(values) || !aligned16(meta) || (ldx % 16) != 0 ||
         (reinterpret_cast<uintptr_t>(X) & 31u) || (reinterpret_cast<uintptr_t>(values) & 31u))
@@ -668,10 +684,10 @@ lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t
         cudaError_t e;
         if (mode == LYNX_COMP_NONE)
             e = cudaLaunchKernelEx(&pc, prune_compress_kernel<false>, Xp, M, K, ldx, vp, mp, row_scale, none_f, none_f,
-                                   none_u, 0, tpu, KS, ctas_per_rb);
+                                   none_u, 0, tpu, KS, ctas_per_rb, 0);
         else
             e = cudaLaunchKernelEx(&pc, prune_compress_kernel<true>, Xp, M, K, ldx, vp, mp, row_scale, sums, partial,
-                                   ctx->tickets, (int)mode, tpu, KS, ctas_per_rb);
+                                   ctx->tickets, (int)mode, tpu, KS, ctas_per_rb, defer ? 1 : 0);
         if (e != cudaSuccess) return LYNX_ERR_CUDA;
     }
     ctx->launches++;
@@ -679,7 +695,16 @@ lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t
         tensor_scale_kernel<<<1, 1024, 0, st>>>(sums, M, row_scale);
         ctx->launches++;
     }
+    if (src) {
+        src->partial = defer ? partial : nullptr;
+        src->ks = defer ? KS : 0;
+    }
     return cuda_ok(cudaGetLastError());
+}
+
+lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, void* values,
+                                void* meta, float* row_scale, lynx_comp_mode mode, void* stream) {
+    return prune_impl(ctx, X, M, K, ldx, values, meta, row_scale, mode, stream, false, nullptr);
 }
 
 lynx_status lynx_sparse_linear(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
@@ -740,13 +765,18 @@ lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int6
     void* values = base + L.values;
     void* meta = base + L.meta;
     float* scale = reinterpret_cast<float*>(base + L.scale);
-    s = lynx_prune_compress(ctx, X, M, K, ldx, values, meta, mode == LYNX_COMP_NONE ? nullptr : scale, mode, stream);
+    // ROW mode: the prune launch stops at its per-K-split row sums and the GEMM's epilogue adds them
+    ScaleSrc ss;
+    s = prune_impl(ctx, X, M, K, ldx, values, meta, mode == LYNX_COMP_NONE ? nullptr : scale, mode, stream,
+                   ctx->defer_scale != 0, &ss);
     if (s != LYNX_OK) return s;
     lynx_comp comp;
-    comp.row_scale = mode == LYNX_COMP_NONE ? nullptr : scale;
+    comp.row_scale = (mode == LYNX_COMP_NONE || ss.partial) ? nullptr : scale;
     comp.residual = residual;
     comp.ldr = ldr;
-    return lynx_sparse_linear(ctx, values, meta, M, K, W, N, ldw, bias, &comp, Y, ldy, stream);
+    if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+    return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &comp, nullptr, Y, ldy,
+                       static_cast<cudaStream_t>(stream), 0, &ss);
 }
 
 lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_host, int64_t M, int64_t K, const void* W,
@@ -856,15 +886,19 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
     void* meta = base + L.meta;
     float* scale = mode == LYNX_COMP_NONE ? nullptr : reinterpret_cast<float*>(base + L.scale);
     void* T = static_cast<char*>(ctx->lora_ws) + LL.T;
-    s = lynx_prune_compress(ctx, X, M, K, ldx, values, meta, scale, mode, stream);
-    if (s != LYNX_OK) return s;
-    lynx_comp comp;
-    comp.row_scale = scale;
-    comp.residual = residual;
-    comp.ldr = ldr;
     const int cfg = pick_gemm_cfg(ctx, M, N, K, (int)(R / 64));
     const bool groups_fit = (size_t)((M + 255) / 256) * 8 * 4 <= L0_WORDS_BYTES;
-    if (ctx->lora_fuse && R == 64 && cfg_supports_l0(cfg) && !ctx->streamk && groups_fit) {
+    const bool fused = ctx->lora_fuse && R == 64 && cfg_supports_l0(cfg) && !ctx->streamk && groups_fit;
+    // (the separate down-projection kernel reads row_scale, so the scale is only deferred when the
+    // GEMM launch is its one consumer)
+    ScaleSrc ss;
+    s = prune_impl(ctx, X, M, K, ldx, values, meta, scale, mode, stream, fused && ctx->defer_scale != 0, &ss);
+    if (s != LYNX_OK) return s;
+    lynx_comp comp;
+    comp.row_scale = ss.partial ? nullptr : scale;
+    comp.residual = residual;
+    comp.ldr = ldr;
+    if (fused) {
         // two launches: the GEMM kernel computes T = (X L_B^T) / s itself before its first tile
         char* ws = static_cast<char*>(ctx->lora_ws);
         LoraArgs lora{T, R, LA, ldla, (int)R};
@@ -876,7 +910,7 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
         lora.l0_tickets = ctx->tickets + (PRUNE_TICKET_BYTES + LORA_TICKET_BYTES) / 4;
         lora.l0_ready = lora.l0_tickets + L0_WORDS_BYTES / 4;
         return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &comp, &lora, Y, ldy,
-                           static_cast<cudaStream_t>(stream), cfg);
+                           static_cast<cudaStream_t>(stream), cfg, &ss);
     }
     s = lynx_lora_down(ctx, X, M, K, ldx, LB, R, ldlb, scale, T, R, stream);
     if (s != LYNX_OK) return s;
@@ -983,11 +1017,11 @@ extern "C" lynx_status lynx_prune_compress_static(const void* X, int64_t M, int6
     if (mode == LYNX_COMP_NONE)
         prune_compress_kernel<false><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
             static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
-            row_scale, nullptr, nullptr, nullptr, 0, tpu, KS, ctas_per_rb);
+            row_scale, nullptr, nullptr, nullptr, 0, tpu, KS, ctas_per_rb, 0);
     else
         prune_compress_kernel<true><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
             static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
-            row_scale, sums, partial, tickets, (int)mode, tpu, KS, ctas_per_rb);
+            row_scale, sums, partial, tickets, (int)mode, tpu, KS, ctas_per_rb, 0);
     if (mode == LYNX_COMP_TENSOR) tensor_scale_kernel<<<1, 1024, 0, st>>>(sums, M, row_scale);
     return cuda_ok(cudaGetLastError());
 }

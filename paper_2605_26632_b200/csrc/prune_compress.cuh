@@ -80,6 +80,29 @@ __device__ __forceinline__ void write_scale_or_sums(int mode, int64_t m, float n
     }
 }
 
+// Row scale from the per-K-split partial sums a deferred prune launch left behind:
+// partial[(row / 16 * KS + ks) * 32 + 2 * (row % 16) + {0: sum x^2, 1: sum kept^2}].  Same order
+// of additions as the in-kernel finalize (eight strided accumulators j = jl, jl + 8, ..., then
+// those eight in ascending order), so both give the same bits.
+__device__ __forceinline__ float row_scale_from_partials(const float* __restrict__ partial, int64_t row, int KS) {
+    const float2* pp = reinterpret_cast<const float2*>(partial) + (row >> 4) * KS * 16 + (row & 15);
+    float n[8], d[8];
+#pragma unroll
+    for (int jl = 0; jl < 8; ++jl) { n[jl] = 0.f; d[jl] = 0.f; }
+    for (int j0 = 0; j0 < KS; j0 += 16) {  // 16 independent loads in flight per round
+        float2 v[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) v[u] = (j0 + u < KS) ? __ldcg(pp + (int64_t)(j0 + u) * 16) : make_float2(0.f, 0.f);
+#pragma unroll
+        for (int u = 0; u < 16; ++u)
+            if (j0 + u < KS) { n[u & 7] += v[u].x; d[u & 7] += v[u].y; }
+    }
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int jl = 0; jl < 8; ++jl) { num += n[jl]; den += d[jl]; }
+    return sqrtf(num / (den + 1e-8f));
+}
+
 // One 32-byte vector = 16 consecutive elements = 4 groups -> 4 value registers + 16 metadata bits.
 __device__ __forceinline__ uint32_t prune_vec16(const uint32_t (&r)[8], const uint32_t* lut,
                                                 uint32_t* v /*[4]*/) {
@@ -181,7 +204,7 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
                       uint16_t* __restrict__ values, uint8_t* __restrict__ meta,
                       float* __restrict__ row_scale, float* __restrict__ sums,
                       float* __restrict__ partial, uint32_t* __restrict__ tickets, int mode,
-                      int tiles_per_unit, int KS, int ctas_per_rb) {
+                      int tiles_per_unit, int KS, int ctas_per_rb, int defer) {
     __shared__ uint32_t lut[4 * 16];
     __shared__ float2 red[PRUNE_CTA_WARPS * 2][16];
     __shared__ uint32_t s_last;
@@ -235,6 +258,17 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
             denA += __shfl_xor_sync(0xffffffffu, denA, off);
             numB += __shfl_xor_sync(0xffffffffu, numB, off);
             denB += __shfl_xor_sync(0xffffffffu, denB, off);
+        }
+        if (defer) {
+            // the consumer (the sparse GEMM's epilogue) adds the partial sums itself, in the order
+            // row_scale_from_partials states: no ticket, no barrier, no fence here
+            if (active) prune_tile_store(last, va, vb, slab, okA, okB);
+            if (active && q == 0) {
+                float* mine = partial + (rb16 * KS + ks) * 32;
+                *reinterpret_cast<float2*>(mine + 2 * r) = make_float2(numA, denA);
+                *reinterpret_cast<float2*>(mine + 2 * (r + 8)) = make_float2(numB, denB);
+            }
+            return;
         }
         if (KS == 1) {
             if (active) prune_tile_store(last, va, vb, slab, okA, okB);

@@ -38,12 +38,15 @@
 #pragma once
 
 #include "ptx.cuh"
+#include "prune_compress.cuh"  // row_scale_from_partials
 
 namespace lynx {
 
 struct GemmParams {
     int64_t M, N, K;
     const float* row_scale;    // [M] or nullptr
+    const float* scale_partial;  // or: per-K-split row sums of a deferred prune launch (see
+    int scale_ks;                //     row_scale_from_partials), scale_ks splits per 16-row block
     const uint16_t* bias;      // [N] bf16 or nullptr
     const uint16_t* residual;  // [M x N] bf16 (ld = ldr) or nullptr
     int64_t ldr;
@@ -530,8 +533,9 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 // the row's scale is fetched while the item's K loop runs (a global load costs over a
                 // microsecond once the main loops saturate the memory system); T = acc * (1 / s)
                 float inv_s = 1.0f;
-                if (p.row_scale != nullptr && row < p.M) {
-                    const float sc = __ldg(p.row_scale + row);
+                if (row < p.M && (p.scale_partial != nullptr || p.row_scale != nullptr)) {
+                    const float sc = (p.scale_partial != nullptr) ? row_scale_from_partials(p.scale_partial, row, p.scale_ks)
+                                                                  : __ldg(p.row_scale + row);
                     inv_s = (sc == 0.0f) ? 0.0f : __frcp_rn(sc);
                 }
                 if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, cta_abort, p.dev_error)) {
@@ -624,12 +628,18 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             const int gi = l0_n + it;
             const int acc = (Cfg::ACC_STAGES == 2) ? (gi & 1) : 0;
             const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((gi >> 1) & 1) : (gi & 1);
-            if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, cta_abort, p.dev_error)) break;
-            tc_fence_after();
             const int m0 = (tm * CG + (int)rank) * Cfg::BM + q * 32;
             const int64_t row = m0 + lane;
             const bool row_ok = row < p.M;
-            const float s = (p.row_scale != nullptr && row_ok) ? p.row_scale[row] : 1.0f;
+            // the row's scale is fetched (or summed from the prune launch's partial sums) while the
+            // tile's main loop still runs
+            float s = 1.0f;
+            if (row_ok) {
+                if (p.scale_partial != nullptr) s = row_scale_from_partials(p.scale_partial, row, p.scale_ks);
+                else if (p.row_scale != nullptr) s = __ldg(p.row_scale + row);
+            }
+            if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, cta_abort, p.dev_error)) break;
+            tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
             // stream-K pieces: this thread's row of the pair tile inside an fp32 partial slot
             const size_t slot_floats = (size_t)Cfg::BM * CG * BN;
