@@ -22,7 +22,7 @@ _LIB = os.path.join(_HERE, "liblynx_oracle.so")
 _lock = threading.Lock()
 _lib = None
 
-COMP_NONE, COMP_ROW, COMP_TENSOR = 0, 1, 2
+COMP_NONE, COMP_ROW, COMP_TENSOR, COMP_GROUP = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -109,6 +109,24 @@ def compress(X: np.ndarray):
     meta = np.empty((M, K // 16), dtype=np.uint16)
     _load().oracle_compress(_p(X), _i64(M), _i64(K), _i64(K), _p(values), _p(meta))
     return values, meta
+
+
+def compress_group_scaled(X: np.ndarray):
+    """Per-group norm compensation folded into the values (fp32 reading).
+    -> (values uint16 [M, K/2] = bf16(s_g * kept), meta_canon uint16 [M, K/16])"""
+    X, M, K = _check_x(X)
+    values = np.empty((M, K // 2), dtype=np.uint16)
+    meta = np.empty((M, K // 16), dtype=np.uint16)
+    _load().oracle_compress_group_scaled(_p(X), _i64(M), _i64(K), _i64(K), _p(values), _p(meta))
+    return values, meta
+
+
+def group_scale_f64(X: np.ndarray) -> np.ndarray:
+    """The per-group factors in fp64: [M, K/4]."""
+    X, M, K = _check_x(X)
+    s = np.empty((M, K // 4), dtype=np.float64)
+    _load().oracle_group_scale_f64(_p(X), _i64(M), _i64(K), _i64(K), _p(s))
+    return s
 
 
 def decompress(values: np.ndarray, meta_canon: np.ndarray) -> np.ndarray:

@@ -119,6 +119,59 @@ ORACLE_API void oracle_compress(const uint16_t* X, int64_t M, int64_t K, int64_t
         }
 }
 
+/* ---- Per-group norm compensation: the literal reading of the norm-compensation equation,
+ * which is written for one group X in R^{1x4}:  S(X) = s * X~,  s = sqrt(|X|^2 / (|X~|^2 + eps)),
+ * eps = 1e-8, with one s per group of four.  A per-group factor cannot be applied after the
+ * product, so it is folded into the stored values: values = bf16_rne(s_g * x_kept).  The paper
+ * fixes no precision for s; the reading taken is fp32 with IEEE operations in this order
+ * (squares of bf16 are exact in fp32, so each line rounds once):
+ *   num = x0^2; num += x1^2; num += x2^2; num += x3^2;      (ascending index)
+ *   den = k0^2; den += k1^2; den += eps;                     (the two kept, ascending index)
+ *   s = sqrtf(num / den);   value_j = bf16_rne(s * k_j)
+ * The mask and the metadata are those of oracle_compress.                                   */
+ORACLE_API void oracle_compress_group_scaled(const uint16_t* X, int64_t M, int64_t K, int64_t ldx,
+                                             uint16_t* values, uint16_t* meta_canon) {
+    const int64_t G = K / 4;
+    memset(meta_canon, 0, (size_t)(M * (K / 16)) * sizeof(uint16_t));
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t g = 0; g < G; ++g) {
+            const uint16_t* grp = X + m * ldx + 4 * g;
+            int i0, i1;
+            select_group(grp, &i0, &i1);
+            float x[4];
+            for (int i = 0; i < 4; ++i) x[i] = bf16_to_f32(grp[i]);
+            float num = x[0] * x[0];
+            num = num + x[1] * x[1];
+            num = num + x[2] * x[2];
+            num = num + x[3] * x[3];
+            float den = x[i0] * x[i0];
+            den = den + x[i1] * x[i1];
+            den = den + 1e-8f;
+            const float sc = sqrtf(num / den);
+            values[m * (K / 2) + 2 * g + 0] = oracle_f32_to_bf16(sc * x[i0]);
+            values[m * (K / 2) + 2 * g + 1] = oracle_f32_to_bf16(sc * x[i1]);
+            unsigned nib = (unsigned)i0 | ((unsigned)i1 << 2);
+            meta_canon[m * (K / 16) + g / 4] |= (uint16_t)(nib << (4 * (g % 4)));
+        }
+}
+
+/* The same factors in fp64, one per group (M x K/4): the check of the fp32 reading above. */
+ORACLE_API void oracle_group_scale_f64(const uint16_t* X, int64_t M, int64_t K, int64_t ldx, double* s) {
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t g = 0; g < K / 4; ++g) {
+            const uint16_t* grp = X + m * ldx + 4 * g;
+            int i0, i1;
+            select_group(grp, &i0, &i1);
+            double num = 0.0, den = 0.0;
+            for (int i = 0; i < 4; ++i) {
+                double x = (double)bf16_to_f32(grp[i]);
+                num += x * x;
+                if (i == i0 || i == i1) den += x * x;
+            }
+            s[m * (K / 4) + g] = sqrt(num / (den + 1e-8));
+        }
+}
+
 /* Step 3: scatter the kept values back; must reproduce mask (.) X bit for bit. */
 ORACLE_API void oracle_decompress(const uint16_t* values, const uint16_t* meta_canon, int64_t M,
                                   int64_t K, uint16_t* Xmasked) {
@@ -188,7 +241,7 @@ ORACLE_API void oracle_meta_hw_to_canon(const uint8_t* meta_hw, int64_t M, int64
 ORACLE_API void oracle_row_scale(const uint16_t* X, int64_t M, int64_t K, int64_t ldx, int mode,
                                  float* s) {
     const double eps = 1e-8;
-    if (mode == 0) {
+    if (mode == 0 || mode == 3) { /* none; per-group factors live in the values, not here */
         for (int64_t m = 0; m < M; ++m) s[m] = 1.0f;
         return;
     }
@@ -334,9 +387,11 @@ ORACLE_API void oracle_act_sparse_linear(const uint16_t* X, int64_t M, int64_t K
                                          int64_t ldr, const int64_t* rows, int64_t n_rows,
                                          uint16_t* values, uint16_t* meta_canon, float* scale_out,
                                          uint16_t* xmasked_scratch, float* acc_scratch, float* Y) {
-    oracle_compress(X, M, K, ldx, values, meta_canon);
+    if (comp_mode == 3) oracle_compress_group_scaled(X, M, K, ldx, values, meta_canon);
+    else oracle_compress(X, M, K, ldx, values, meta_canon);
     oracle_decompress(values, meta_canon, M, K, xmasked_scratch);
     oracle_row_scale(X, M, K, ldx, comp_mode, scale_out);
     oracle_gemm_masked_f32(xmasked_scratch, K, W, N, ldw, rows, n_rows, acc_scratch);
-    oracle_epilogue(acc_scratch, N, rows, n_rows, comp_mode ? scale_out : NULL, bias, Yr, ldr, Y);
+    oracle_epilogue(acc_scratch, N, rows, n_rows, (comp_mode == 1 || comp_mode == 2) ? scale_out : NULL, bias, Yr,
+                    ldr, Y);
 }

@@ -326,6 +326,87 @@ def test_lora_residual_matches_library_matmul():
     np.testing.assert_allclose(got, ref.numpy(), rtol=1e-5, atol=1e-6)
 
 
+# ---------------------------------------------------------------- per-group norm compensation ---
+
+def _bf(vals):
+    return inputs.as_u16(torch.tensor(vals, dtype=torch.float32).to(torch.bfloat16).reshape(1, -1))
+
+
+def test_group_scale_closed_forms():
+    """[a,a,a,a] keeps two of four equal squares: s = sqrt(2); a group that already has two zeros
+    keeps everything: s = 1 and the values are bit copies; a zero group stays zero."""
+    x = _bf([1, 1, 1, 1, 3, 4, 0, 0, 0, 0, 0, 0, -2, 0.5, 0.25, 2])
+    x = np.tile(x, (1, 8))  # K = 128
+    v, meta = oracle.compress_group_scaled(x)
+    v0, meta0 = oracle.compress(x)
+    assert (meta == meta0).all()
+    got = inputs.from_u16(v).float().numpy()[0, :8]
+    sqrt2 = float(torch.tensor(2.0 ** 0.5).to(torch.bfloat16))
+    assert got[0] == sqrt2 and got[1] == sqrt2
+    assert got[2] == 3.0 and got[3] == 4.0
+    assert got[4] == 0.0 and got[5] == 0.0
+    # [-2, .5, .25, 2]: kept -2 and 2, s = sqrt(8.3125 / 8)
+    s = (8.3125 / 8.0) ** 0.5
+    ref = torch.tensor([-2 * s, 2 * s]).to(torch.bfloat16).float().numpy()
+    assert got[6] == ref[0] and got[7] == ref[1]
+
+
+def test_group_scale_restores_each_groups_norm_and_matches_fp64():
+    g = torch.Generator().manual_seed(21)
+    M, K = 64, 512
+    x = (torch.randn(M, K, generator=g) * torch.exp(torch.randn(M, K, generator=g))).to(torch.bfloat16)
+    X = inputs.as_u16(x)
+    v, meta = oracle.compress_group_scaled(X)
+    v0, _ = oracle.compress(X)
+    vs = inputs.from_u16(v).double().numpy().reshape(M, K // 4, 2)
+    kept = inputs.from_u16(v0).double().numpy().reshape(M, K // 4, 2)
+    xs = x.double().numpy().reshape(M, K // 4, 4)
+    # the scaled pair carries the group's whole norm (up to the bf16 rounding of two values)
+    np.testing.assert_allclose((vs ** 2).sum(-1), (xs ** 2).sum(-1), rtol=2.0 ** -7, atol=1e-7)
+    # the fp32 reading agrees with the fp64 factors to within one bf16 step, and almost always exactly
+    s64 = oracle.group_scale_f64(X)
+    ref = torch.from_numpy(kept * s64[..., None]).to(torch.bfloat16).double().numpy()
+    assert (np.abs(vs - ref) <= np.abs(ref) * 2.0 ** -7).all()
+    assert (vs == ref).mean() > 0.995
+    # a scale >= 1 never shrinks a kept value, and it is at most sqrt(2) for Top-2-of-4... of equal
+    # magnitudes; in general at most 2 (two kept carry at least half of four squares only when
+    # they are the largest two, which they are): |X|^2 <= 2 |X~|^2
+    assert (s64 <= 2.0 ** 0.5 + 1e-6).all() and (s64[(xs ** 2).sum(-1) > 1e-6] >= 1.0 - 1e-6).all()
+
+
+def test_group_mode_equals_row_mode_when_a_row_is_one_group():
+    """K = 128 is the smallest K; make 31 of the 32 groups of every row zero: then the row scale
+    and the only non-zero group's scale are the same number."""
+    g = torch.Generator().manual_seed(22)
+    M, K = 48, 128
+    x = torch.zeros(M, K)
+    x[:, 8:12] = torch.randn(M, 4, generator=g)
+    x = x.to(torch.bfloat16)
+    X = inputs.as_u16(x)
+    v, _ = oracle.compress_group_scaled(X)
+    v0, _ = oracle.compress(X)
+    s_row = oracle.row_scale(X, oracle.COMP_ROW).astype(np.float64)
+    ref = torch.from_numpy(inputs.from_u16(v0).double().numpy() * s_row[:, None]).to(torch.bfloat16).double().numpy()
+    got = inputs.from_u16(v).double().numpy()
+    assert (np.abs(got - ref) <= np.abs(ref) * 2.0 ** -7).all()
+    assert (got == ref).mean() > 0.99
+
+
+def test_group_mode_whole_path_is_the_product_of_the_scaled_sparse_activation():
+    g = torch.Generator().manual_seed(23)
+    M, K, N = 16, 256, 40
+    x = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    w = (torch.randn(N, K, generator=g) * K ** -0.5).to(torch.bfloat16)
+    b = (torch.randn(N, generator=g) * 0.1).to(torch.bfloat16)
+    out = oracle.act_sparse_linear(inputs.as_u16(x), inputs.as_u16(w), bias=inputs.as_u16(b), comp_mode=oracle.COMP_GROUP)
+    v, meta = oracle.compress_group_scaled(inputs.as_u16(x))
+    assert (out["values"] == v).all() and (out["meta_canon"] == meta).all()
+    xs = inputs.from_u16(oracle.decompress(v, meta)).double()
+    ref = xs @ w.double().T + b.double()
+    np.testing.assert_allclose(out["Y"], ref.numpy(), rtol=1e-4, atol=1e-5)
+    assert (out["scale"] == 1.0).all()
+
+
 def test_lora_rows_subset_equals_full_rows():
     g = torch.Generator().manual_seed(12)
     M, K, R, N = 20, 128, 8, 24
