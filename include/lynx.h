@@ -59,7 +59,9 @@ typedef enum {
 typedef enum {
     LYNX_COMP_NONE = 0,  /* no rescaling: y = x~ W^T + b  (Algorithm 2, activation_sparse)   */
     LYNX_COMP_ROW = 1,   /* one s per token row (the reading used by default)                */
-    LYNX_COMP_TENSOR = 2 /* one s for the whole X (Algorithm 1 read literally)               */
+    LYNX_COMP_TENSOR = 2, /* one s for the whole X (Algorithm 1 read literally)              */
+    LYNX_COMP_GROUP = 3   /* one s per group of four (the norm-compensation equation read
+                             literally): folded into the stored values, see lynx_prune_compress */
 } lynx_comp_mode;
 
 typedef enum {
@@ -113,6 +115,11 @@ LYNX_API lynx_status lynx_reserve(lynx_ctx* ctx, int64_t M, int64_t N, int64_t K
  *         row-major form for inspection.
  *   row_scale (may be NULL when mode == LYNX_COMP_NONE): [M] fp32, s_m per `mode`
  *         (ROW: per row; TENSOR: the same global s in every entry; NONE: 1.0 if non-NULL).
+ * LYNX_COMP_GROUP: values[m, 2g+j] = bf16_rne( s_{m,g} * X[m, 4g + idx_j] ) with, in fp32 and IEEE
+ *         operations in this order, num = ((x0^2 + x1^2) + x2^2) + x3^2, den = (k0^2 + k1^2) + 1e-8
+ *         (k = the two kept elements), s = sqrt(num / den); metadata as in every mode; row_scale,
+ *         if given, is written as 1.0 and the product that follows needs no scale.  (Not
+ *         available with LYNX_FUSE_FUSED.)
  * Alignment for this step: X and values 32-byte aligned, ldx % 16 == 0 (32-byte vector
  * accesses), meta 16-byte aligned; violations return LYNX_ERR_ALIGNMENT.
  * ROW and TENSOR modes use the context's scratch: partial sums of each 16-row block per run of

@@ -14,7 +14,7 @@ import torch
 
 from . import build as _build
 
-COMP_NONE, COMP_ROW, COMP_TENSOR = 0, 1, 2
+COMP_NONE, COMP_ROW, COMP_TENSOR, COMP_GROUP = 0, 1, 2, 3
 FUSE_AUTO, FUSE_SEPARATE, FUSE_FUSED = 0, 1, 2
 
 EXPORTS = [
@@ -133,7 +133,7 @@ def prune_compress_static(X: torch.Tensor, mode: int = COMP_NONE, values=None, m
         values = torch.empty((M, K // 2), dtype=torch.bfloat16, device=X.device)
     if meta is None:
         meta = torch.empty(meta_bytes(M, K), dtype=torch.uint8, device=X.device)
-    if row_scale is None and mode != COMP_NONE:
+    if row_scale is None and mode in (COMP_ROW, COMP_TENSOR):
         row_scale = torch.empty(M, dtype=torch.float32, device=X.device)
     _check(load_library().lynx_prune_compress_static(_ptr(X), M, K, X.stride(0), _ptr(values), _ptr(meta),
                                                      _ptr(row_scale), mode, _stream()),
@@ -181,7 +181,7 @@ class Lynx:
             values = torch.empty((M, K // 2), dtype=torch.bfloat16, device=X.device)
         if meta is None:
             meta = torch.empty(meta_bytes(M, K), dtype=torch.uint8, device=X.device)
-        if row_scale is None and mode != COMP_NONE:
+        if row_scale is None and mode in (COMP_ROW, COMP_TENSOR):
             row_scale = torch.empty(M, dtype=torch.float32, device=X.device)
         _check(self._lib.lynx_prune_compress(self._h, _ptr(X), M, K, X.stride(0), _ptr(values), _ptr(meta),
                                              _ptr(row_scale), mode, _stream()), "lynx_prune_compress")

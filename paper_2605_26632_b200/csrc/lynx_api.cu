@@ -625,15 +625,18 @@ int64_t lynx_launch_count(lynx_ctx* ctx) { return ctx ? ctx->launches : -1; }
 // The prune/compress launch.  defer (ROW mode only): the kernel stops at the per-K-split row sums
 // and `src` tells the following GEMM where they are; its epilogue adds them in the same order the
 // in-kernel finalize would (same bits), which saves the ticket hand-over inside this kernel.
+static bool sums_needed(lynx_comp_mode mode) { return mode == LYNX_COMP_ROW || mode == LYNX_COMP_TENSOR; }
+
 static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, void* values,
                               void* meta, float* row_scale, lynx_comp_mode mode, void* stream, bool defer,
                               ScaleSrc* src) {
     lynx_status s = check_common(ctx, M, K);
     if (s != LYNX_OK) return s;
     if (!X || !values || !meta) return LYNX_ERR_INVALID_ARG;
-    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW && mode != LYNX_COMP_TENSOR) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW && mode != LYNX_COMP_TENSOR && mode != LYNX_COMP_GROUP)
+        return LYNX_ERR_INVALID_ARG;
     if (mode != LYNX_COMP_ROW) defer = false;
-    if (mode != LYNX_COMP_NONE && !row_scale && !defer) return LYNX_ERR_INVALID_ARG;
+    if (sums_needed(mode) && !row_scale && !defer) return LYNX_ERR_INVALID_ARG;
     if (ldx < K) return LYNX_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(values) || !aligned16(meta) || (ldx % 16) != 0 ||
         (reinterpret_cast<uintptr_t>(X) & 31u) || (reinterpret_cast<uintptr_t>(values) & 31u))
@@ -653,7 +656,7 @@ static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
     const int KS = (int)(kblocks / tpu);
     float* sums = nullptr;
     float* partial = nullptr;
-    if (mode != LYNX_COMP_NONE) {
+    if (sums_needed(mode)) {
         std::lock_guard<std::mutex> lock(ctx->mu);
         ScratchLayout L = scratch_layout(M, 8, K);
         if (ctx->scratch_bytes < L.prune_end) {
@@ -683,10 +686,13 @@ static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
         uint32_t* none_u = nullptr;
         cudaError_t e;
         if (mode == LYNX_COMP_NONE)
-            e = cudaLaunchKernelEx(&pc, prune_compress_kernel<false>, Xp, M, K, ldx, vp, mp, row_scale, none_f, none_f,
-                                   none_u, 0, tpu, KS, ctas_per_rb, 0);
+            e = cudaLaunchKernelEx(&pc, prune_compress_kernel<false, false>, Xp, M, K, ldx, vp, mp, row_scale, none_f,
+                                   none_f, none_u, 0, tpu, KS, ctas_per_rb, 0);
+        else if (mode == LYNX_COMP_GROUP)
+            e = cudaLaunchKernelEx(&pc, prune_compress_kernel<false, true>, Xp, M, K, ldx, vp, mp, row_scale, none_f,
+                                   none_f, none_u, 0, tpu, KS, ctas_per_rb, 0);
         else
-            e = cudaLaunchKernelEx(&pc, prune_compress_kernel<true>, Xp, M, K, ldx, vp, mp, row_scale, sums, partial,
+            e = cudaLaunchKernelEx(&pc, prune_compress_kernel<true, false>, Xp, M, K, ldx, vp, mp, row_scale, sums, partial,
                                    ctx->tickets, (int)mode, tpu, KS, ctas_per_rb, defer ? 1 : 0);
         if (e != cudaSuccess) return LYNX_ERR_CUDA;
     }
@@ -737,7 +743,8 @@ lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int6
     if (N < 8) return LYNX_ERR_INVALID_ARG;
     if (fuse == LYNX_FUSE_FUSED) {
         // the whole-tensor scale needs all of X before the first output: two-kernel path only
-        if (mode == LYNX_COMP_TENSOR) return LYNX_ERR_UNSUPPORTED_SHAPE;
+        // (and the per-group factors are only built into the stand-alone prune kernel)
+        if (mode == LYNX_COMP_TENSOR || mode == LYNX_COMP_GROUP) return LYNX_ERR_UNSUPPORTED_SHAPE;
         if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW) return LYNX_ERR_INVALID_ARG;
         if (!X || !W || !Y) return LYNX_ERR_INVALID_ARG;
         if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
@@ -767,11 +774,11 @@ lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int6
     float* scale = reinterpret_cast<float*>(base + L.scale);
     // ROW mode: the prune launch stops at its per-K-split row sums and the GEMM's epilogue adds them
     ScaleSrc ss;
-    s = prune_impl(ctx, X, M, K, ldx, values, meta, mode == LYNX_COMP_NONE ? nullptr : scale, mode, stream,
+    s = prune_impl(ctx, X, M, K, ldx, values, meta, sums_needed(mode) ? scale : nullptr, mode, stream,
                    ctx->defer_scale != 0, &ss);
     if (s != LYNX_OK) return s;
     lynx_comp comp;
-    comp.row_scale = (mode == LYNX_COMP_NONE || ss.partial) ? nullptr : scale;
+    comp.row_scale = (!sums_needed(mode) || ss.partial) ? nullptr : scale;
     comp.residual = residual;
     comp.ldr = ldr;
     if ((s = check_device_error(ctx)) != LYNX_OK) return s;
@@ -884,7 +891,7 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
     char* base = static_cast<char*>(ctx->scratch);
     void* values = base + L.values;
     void* meta = base + L.meta;
-    float* scale = mode == LYNX_COMP_NONE ? nullptr : reinterpret_cast<float*>(base + L.scale);
+    float* scale = sums_needed(mode) ? reinterpret_cast<float*>(base + L.scale) : nullptr;
     void* T = static_cast<char*>(ctx->lora_ws) + LL.T;
     const int cfg = pick_gemm_cfg(ctx, M, N, K, (int)(R / 64));
     const bool groups_fit = (size_t)((M + 255) / 256) * 8 * 4 <= L0_WORDS_BYTES;
@@ -982,8 +989,9 @@ extern "C" lynx_status lynx_prune_compress_static(const void* X, int64_t M, int6
     if (M < 1 || K < 128) return LYNX_ERR_INVALID_ARG;
     if (K % 128 != 0 || M > (1ll << 30) || K > (1ll << 30)) return LYNX_ERR_UNSUPPORTED_SHAPE;
     if (!X || !values || !meta) return LYNX_ERR_INVALID_ARG;
-    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW && mode != LYNX_COMP_TENSOR) return LYNX_ERR_INVALID_ARG;
-    if (mode != LYNX_COMP_NONE && !row_scale) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW && mode != LYNX_COMP_TENSOR && mode != LYNX_COMP_GROUP)
+        return LYNX_ERR_INVALID_ARG;
+    if (sums_needed(mode) && !row_scale) return LYNX_ERR_INVALID_ARG;
     if (ldx < K) return LYNX_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(X) & 31u) || (reinterpret_cast<uintptr_t>(values) & 31u) || !aligned16(meta) ||
         (ldx % 16) != 0)
@@ -1004,7 +1012,7 @@ extern "C" lynx_status lynx_prune_compress_static(const void* X, int64_t M, int6
     // (a __device__ array starts zeroed and every launch leaves its tickets at zero again)
     constexpr size_t STATIC_TICKET_BYTES = 64u << 10;
     if ((size_t)rb16 * 4 > STATIC_TICKET_BYTES) return LYNX_ERR_WORKSPACE;
-    const size_t partial_bytes = (mode != LYNX_COMP_NONE && KS > 1) ? (size_t)rb16 * KS * 32 * 4 : 0;
+    const size_t partial_bytes = (sums_needed(mode) && KS > 1) ? (size_t)rb16 * KS * 32 * 4 : 0;
     const size_t partial_padded = (partial_bytes + 255) / 256 * 256;
     const size_t sums_bytes = (mode == LYNX_COMP_TENSOR) ? (size_t)M * 8 : 0;
     if (STATIC_TICKET_BYTES + partial_padded + sums_bytes > (size_t)LYNX_STATIC_SCRATCH_BYTES) return LYNX_ERR_WORKSPACE;
@@ -1014,7 +1022,11 @@ extern "C" lynx_status lynx_prune_compress_static(const void* X, int64_t M, int6
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int ctas_per_rb = (KS + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS;
     const unsigned grid = (unsigned)(rb16 * ctas_per_rb);
-    if (mode == LYNX_COMP_NONE)
+    if (mode == LYNX_COMP_GROUP)
+        prune_compress_kernel<false, true><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
+            static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
+            row_scale, nullptr, nullptr, nullptr, 0, tpu, KS, ctas_per_rb, 0);
+    else if (mode == LYNX_COMP_NONE)
         prune_compress_kernel<false><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
             static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),
             row_scale, nullptr, nullptr, nullptr, 0, tpu, KS, ctas_per_rb, 0);

@@ -120,6 +120,32 @@ __device__ __forceinline__ uint32_t prune_vec16(const uint32_t (&r)[8], const ui
     return (e0 | e1 | e2 | e3) >> 16;
 }
 
+// Per-group norm compensation (the norm-compensation equation read literally, one s per group of
+// four): v holds the group's two kept bf16 (lower index in the lower half), r01 / r23 its four
+// elements.  fp32, IEEE operations, in this order:
+// num = ((x0^2 + x1^2) + x2^2) + x3^2;  den = (k0^2 + k1^2) + 1e-8;
+// s = sqrt(num / den);  result = bf16_rne(s * k0), bf16_rne(s * k1).
+__device__ __forceinline__ uint32_t group_scale_pair(uint32_t r01, uint32_t r23, uint32_t v) {
+    const float x0 = bf16_lo_f(r01), x1 = bf16_hi_f(r01), x2 = bf16_lo_f(r23), x3 = bf16_hi_f(r23);
+    const float k0 = bf16_lo_f(v), k1 = bf16_hi_f(v);
+    // (separately rounded products and sums, never fused: a square that underflows rounds the
+    // same way on every machine)
+    float num = __fmul_rn(x0, x0);
+    num = __fadd_rn(num, __fmul_rn(x1, x1));
+    num = __fadd_rn(num, __fmul_rn(x2, x2));
+    num = __fadd_rn(num, __fmul_rn(x3, x3));
+    float den = __fmul_rn(k0, k0);
+    den = __fadd_rn(den, __fmul_rn(k1, k1));
+    den = __fadd_rn(den, 1e-8f);
+    const float sc = __fsqrt_rn(__fdiv_rn(num, den));
+    return pack_bf16x2(__fmul_rn(sc, k0), __fmul_rn(sc, k1));
+}
+
+__device__ __forceinline__ void group_scale_vec16(const uint32_t (&r)[8], uint32_t* v /*[4]*/) {
+#pragma unroll
+    for (int g = 0; g < 4; ++g) v[g] = group_scale_pair(r[2 * g], r[2 * g + 1], v[g]);
+}
+
 // Work unit of one warp: 16 rows x (tiles_per_unit * 128) elements; the KS = kblocks /
 // tiles_per_unit units of a 16-row block are independent warps (many small CTAs keep the SMs'
 // load queues full).  With KS > 1 each unit writes its partial row sums
@@ -127,7 +153,8 @@ __device__ __forceinline__ uint32_t prune_vec16(const uint32_t (&r)[8], const ui
 // block to finish adds them in a fixed order, so the result does not depend on scheduling.
 //
 // mode: 0 none (row_scale written as 1 if non-null), 1 per-row scale, 2 per-row sums for the
-// whole-tensor scale (sums[2*m] = sum x^2, sums[2*m+1] = sum kept x^2).
+// whole-tensor scale (sums[2*m] = sum x^2, sums[2*m+1] = sum kept x^2).  GROUP (with SUMS = false):
+// the kept values are stored multiplied by their group's factor (group_scale_pair).
 #ifndef LYNX_PRUNE_CTA_WARPS
 #define LYNX_PRUNE_CTA_WARPS 4
 #endif
@@ -142,7 +169,7 @@ struct TileOut {
     uint32_t w0, w1;        // the lane's two metadata words
 };
 
-template <bool SUMS, bool GUARD>
+template <bool SUMS, bool GUARD, bool GROUP = false>
 __device__ __forceinline__ void prune_tile_compute(const uint16_t* xa, const uint16_t* xb, bool okA, bool okB,
                                                    const uint32_t* lut, TileOut& out, float& numA, float& denA,
                                                    float& numB, float& denB) {
@@ -168,6 +195,12 @@ __device__ __forceinline__ void prune_tile_compute(const uint16_t* xa, const uin
     const uint32_t ma1 = prune_vec16(a1, lut, out.oa + 4);
     const uint32_t mb0 = prune_vec16(b0, lut, out.ob);
     const uint32_t mb1 = prune_vec16(b1, lut, out.ob + 4);
+    if constexpr (GROUP) {
+        group_scale_vec16(a0, out.oa);
+        group_scale_vec16(a1, out.oa + 4);
+        group_scale_vec16(b0, out.ob);
+        group_scale_vec16(b1, out.ob + 4);
+    }
     // rows past M prune to the pattern (0,1) = nibble 0x4, the documented padding
     out.w0 = ma0 | (mb0 << 16);
     out.w1 = ma1 | (mb1 << 16);
@@ -198,7 +231,7 @@ __device__ __forceinline__ void prune_tile_store(const TileOut& out, uint16_t* v
     slab[32] = out.w1;
 }
 
-template <bool SUMS>
+template <bool SUMS, bool GROUP = false>
 __global__ void __launch_bounds__(PRUNE_CTA_WARPS * 32, LYNX_PRUNE_MIN_CTAS)
 prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int64_t ldx,
                       uint16_t* __restrict__ values, uint8_t* __restrict__ meta,
@@ -240,9 +273,9 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
         vb = va + 8 * (K / 2);
         for (int t = 0; t < tiles_per_unit; ++t) {
             if (full_rows)
-                prune_tile_compute<SUMS, false>(xa, xb, true, true, lut, last, numA, denA, numB, denB);
+                prune_tile_compute<SUMS, false, GROUP>(xa, xb, true, true, lut, last, numA, denA, numB, denB);
             else
-                prune_tile_compute<SUMS, true>(xa, xb, okA, okB, lut, last, numA, denA, numB, denB);
+                prune_tile_compute<SUMS, true, GROUP>(xa, xb, okA, okB, lut, last, numA, denA, numB, denB);
             if (t + 1 < tiles_per_unit) {
                 prune_tile_store(last, va, vb, slab, okA, okB);
                 xa += 128; xb += 128; va += 64; vb += 64; slab += 512;
