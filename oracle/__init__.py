@@ -241,6 +241,66 @@ def lora_residual(X, LB, LA, rows=None) -> np.ndarray:
     return Yr
 
 
+# ------------------------------------------------------------------------- FP8 composition ---
+
+def e4m3_encode(x) -> np.ndarray:
+    """fp32 -> E4M3 (FN) codes: round to nearest even, finite overflow and Inf saturate to +-448."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint8)
+    _load().oracle_e4m3_encode_array(_p(x), _i64(x.size), _p(out))
+    return out
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    lib = _load()
+    lib.oracle_e4m3_decode.restype = ctypes.c_float
+    lib.oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+    table = np.array([lib.oracle_e4m3_decode(i) for i in range(256)], dtype=np.float32)
+    return table[np.asarray(codes, dtype=np.uint8)]
+
+
+def quantize_weights_fp8(W, per_channel: bool):
+    """-> (Wq uint8 [N, K], wscale float32 [N]); per_channel False = direct cast (scale 1)."""
+    W = _u16(W, "W")
+    N, K = W.shape
+    Wq = np.empty((N, K), dtype=np.uint8)
+    ws = np.empty(N, dtype=np.float32)
+    _load().oracle_quantize_weights_fp8(_p(W), _i64(N), _i64(K), _i64(K), ctypes.c_int(1 if per_channel else 0),
+                                        _p(Wq), _p(ws))
+    return Wq, ws
+
+
+def compress_fp8(X):
+    """-> (values_q uint8 [M, K/2], meta_canon uint16 [M, K/16], act_scale float32 [M])"""
+    X, M, K = _check_x(X)
+    vq = np.empty((M, K // 2), dtype=np.uint8)
+    meta = np.empty((M, K // 16), dtype=np.uint16)
+    sc = np.empty(M, dtype=np.float32)
+    _load().oracle_compress_fp8(_p(X), _i64(M), _i64(K), _i64(K), _p(vq), _p(meta), _p(sc))
+    return vq, meta, sc
+
+
+def act_sparse_linear_fp8(X, Wq, wscale, bias=None, comp_mode=COMP_NONE, Yr=None, rows=None):
+    """Whole FP8 path.  -> dict(values_q, meta_canon, row_scale (= s * act_scale), Y[fp32, rows x N])."""
+    X, M, K = _check_x(X)
+    Wq = np.ascontiguousarray(Wq, dtype=np.uint8)
+    wscale = np.ascontiguousarray(wscale, dtype=np.float32)
+    N = Wq.shape[0]
+    assert Wq.shape == (N, K) and wscale.shape == (N,) and comp_mode in (COMP_NONE, COMP_ROW)
+    bias = None if bias is None else _u16(bias, "bias")
+    Yr = None if Yr is None else _u16(Yr, "Yr")
+    r, nr = _rows(rows, M)
+    vq = np.empty((M, K // 2), dtype=np.uint8)
+    meta = np.empty((M, K // 16), dtype=np.uint16)
+    rs = np.empty(M, dtype=np.float32)
+    acc = np.empty((nr, N), dtype=np.float32)
+    Y = np.empty((nr, N), dtype=np.float32)
+    _load().oracle_act_sparse_linear_fp8(_p(X), _i64(M), _i64(K), _i64(K), _p(Wq), _p(wscale), _i64(N), _p(bias),
+                                         ctypes.c_int(comp_mode), _p(Yr), _i64(N), _p(r), _i64(nr), _p(vq),
+                                         _p(meta), _p(rs), _p(acc), _p(Y))
+    return {"values_q": vq, "meta_canon": meta, "row_scale": rs, "Y": Y}
+
+
 def act_sparse_linear_lora(X, W, LA, LB, bias=None, comp_mode=COMP_NONE, Yr=None, rows=None):
     """Whole path of Algorithm 1 with the LoRA branch: Y = s * (X~ W^T) + b [+ Yr] + X (L_A L_B)^T."""
     out = act_sparse_linear(X, W, bias=bias, comp_mode=comp_mode, Yr=Yr, rows=rows)

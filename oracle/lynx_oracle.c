@@ -24,6 +24,7 @@
 #include <math.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 #define ORACLE_API __attribute__((visibility("default")))
@@ -394,4 +395,166 @@ ORACLE_API void oracle_act_sparse_linear(const uint16_t* X, int64_t M, int64_t K
     oracle_gemm_masked_f32(xmasked_scratch, K, W, N, ldw, rows, n_rows, acc_scratch);
     oracle_epilogue(acc_scratch, N, rows, n_rows, (comp_mode == 1 || comp_mode == 2) ? scale_out : NULL, bias, Yr,
                     ldr, Y);
+}
+
+/* ======================================================================================== *
+ * FP8 composition (the paper's W8A8 compatibility experiment: symmetric FP8 quantisation of
+ * the activations, weights cast to FP8, the 2:4 pattern on FP8 operands).
+ *
+ * FP8 here is E4M3 in the OCP "FN" flavour: 1 sign, 4 exponent bits (bias 7), 3 mantissa bits,
+ * no infinities, S.1111.111 is NaN, largest finite 448, smallest subnormal 2^-9.
+ * The paper fixes neither the granularity of the activation scale nor any rounding; the
+ * reading taken (and restated in the CUDA library's header) is:
+ *   selection      on the bf16 activations, as everywhere else (the mask does not change);
+ *   activation     per token row m: amax_m = max |x~| over the kept values (= max over the row),
+ *                  inv_m = 448 / amax_m (fp32 division; 0 if amax_m = 0),
+ *                  code = e4m3_rne_satfinite(x~ * inv_m)  (fp32 product, then one rounding),
+ *                  act_scale_m = amax_m / 448 (fp32 division);
+ *   weights        "direct": code = e4m3_rne_satfinite(w), w_scale_n = 1; or per output channel:
+ *                  the same symmetric rule over row n of W;
+ *   product        fp32 accumulation of the decoded codes;
+ *   epilogue       y = (s_m * act_scale_m) * w_scale_n * acc + bias + Y_r, s_m the per-row norm
+ *                  compensation of the bf16 activations (1 in mode none).
+ * ======================================================================================== */
+
+ORACLE_API float oracle_e4m3_decode(uint8_t c) {
+    const int sign = c >> 7, e = (c >> 3) & 0xf, m = c & 7;
+    float v;
+    if (e == 0xf && m == 7) v = NAN;
+    else if (e == 0) v = ldexpf((float)m, -9);              /* subnormal: m * 2^-9 */
+    else v = ldexpf((float)(8 + m), e - 7 - 3);             /* (1 + m/8) * 2^(e-7) */
+    return sign ? -v : v;
+}
+
+/* fp32 -> E4M3, round to nearest even, finite overflow (and +-Inf) saturates to +-448, NaN -> 0x7f | sign */
+ORACLE_API uint8_t oracle_e4m3_encode(float f) {
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    const uint8_t sign = (uint8_t)((u >> 24) & 0x80u);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint8_t)(sign | 0x7fu);
+    const float a = fabsf(f);
+    if (!(a < 464.0f)) return (uint8_t)(sign | 0x7eu);       /* >= halfway between 448 and 480: max finite */
+    /* the E4M3 grid around a: spacing 2^(e-3) for normal exponents e = floor(log2 a) >= -6, 2^-9 below */
+    int e;
+    (void)frexpf(a, &e);                                      /* a = f * 2^e, f in [0.5, 1) */
+    int ex = e - 1;                                           /* floor(log2 a) for a > 0 */
+    if (a == 0.0f || ex < -6) ex = -6;
+    const float step = ldexpf(1.0f, ex - 3);
+    /* a / step is exact (power-of-two scaling of a number with more bits than needed is only
+     * exact when no bits fall off the bottom: a has 24 bits, the quotient is < 16, so bits can
+     * fall off only below 2^-20 of a unit -- rintf sees the exact value's neighbourhood; to stay
+     * exact the quotient is formed in double) */
+    const double q = (double)a / (double)step;
+    double r = nearbyint(q);                                  /* current mode: to nearest even */
+    if (r * (double)step > 448.0) r = 448.0 / (double)step;   /* cannot happen after the 464 test; kept for clarity */
+    const float qv = (float)(r * (double)step);               /* the rounded magnitude, exactly representable */
+    /* encode qv */
+    if (qv == 0.0f) return sign;
+    int e2;
+    const float fr = frexpf(qv, &e2);                         /* qv = fr * 2^e2, fr in [0.5,1) */
+    int ee = e2 - 1;                                          /* floor(log2 qv) */
+    uint8_t code;
+    if (ee < -6) code = (uint8_t)lrintf(ldexpf(qv, 9));       /* subnormal: m = qv * 2^9 */
+    else code = (uint8_t)(((ee + 7) << 3) | ((int)lrintf(ldexpf(fr, 4)) - 8)); /* fr*2 in [1,2): m = (fr*2 - 1) * 8 */
+    return (uint8_t)(sign | code);
+}
+
+ORACLE_API void oracle_e4m3_encode_array(const float* in, int64_t n, uint8_t* out) {
+    for (int64_t i = 0; i < n; ++i) out[i] = oracle_e4m3_encode(in[i]);
+}
+
+/* Weights: mode 0 direct cast, 1 symmetric per output channel.  Wq is N x K codes, wscale N floats. */
+ORACLE_API void oracle_quantize_weights_fp8(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode,
+                                            uint8_t* Wq, float* wscale) {
+    for (int64_t n = 0; n < N; ++n) {
+        float inv = 1.0f, sc = 1.0f;
+        if (mode == 1) {
+            float amax = 0.0f;
+            for (int64_t k = 0; k < K; ++k) {
+                float a = fabsf(bf16_to_f32(W[n * ldw + k]));
+                if (a > amax) amax = a;                        /* NaN never raises the maximum */
+            }
+            inv = amax > 0.0f ? 448.0f / amax : 0.0f;
+            sc = amax / 448.0f;
+        }
+        for (int64_t k = 0; k < K; ++k) Wq[n * K + k] = oracle_e4m3_encode(bf16_to_f32(W[n * ldw + k]) * inv);
+        wscale[n] = sc;
+    }
+}
+
+/* Activations: Top-2-of-4 on the bf16 values, then per-row symmetric FP8 codes of the kept ones.
+ * values_q [M x K/2] codes, meta_canon as oracle_compress, act_scale [M]. */
+ORACLE_API void oracle_compress_fp8(const uint16_t* X, int64_t M, int64_t K, int64_t ldx, uint8_t* values_q,
+                                    uint16_t* meta_canon, float* act_scale) {
+    const int64_t G = K / 4;
+    memset(meta_canon, 0, (size_t)(M * (K / 16)) * sizeof(uint16_t));
+    for (int64_t m = 0; m < M; ++m) {
+        float amax = 0.0f;
+        for (int64_t k = 0; k < K; ++k) {
+            float a = fabsf(bf16_to_f32(X[m * ldx + k]));
+            if (a > amax) amax = a;
+        }
+        const float inv = amax > 0.0f ? 448.0f / amax : 0.0f;
+        act_scale[m] = amax / 448.0f;
+        for (int64_t g = 0; g < G; ++g) {
+            const uint16_t* grp = X + m * ldx + 4 * g;
+            int i0, i1;
+            select_group(grp, &i0, &i1);
+            values_q[m * (K / 2) + 2 * g + 0] = oracle_e4m3_encode(bf16_to_f32(grp[i0]) * inv);
+            values_q[m * (K / 2) + 2 * g + 1] = oracle_e4m3_encode(bf16_to_f32(grp[i1]) * inv);
+            unsigned nib = (unsigned)i0 | ((unsigned)i1 << 2);
+            meta_canon[m * (K / 16) + g / 4] |= (uint16_t)(nib << (4 * (g % 4)));
+        }
+    }
+}
+
+/* Product of the decoded codes, fp32 accumulation, k ascending, for the listed rows. */
+ORACLE_API void oracle_gemm_fp8_f32(const uint8_t* values_q, const uint16_t* meta_canon, int64_t M, int64_t K,
+                                    const uint8_t* Wq, int64_t N, const int64_t* rows, int64_t n_rows, float* acc) {
+    if (!rows) n_rows = M;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < n_rows; ++i) {
+        const int64_t m = rows ? rows[i] : i;
+        float* xrow = (float*)malloc((size_t)K * sizeof(float));
+        for (int64_t k = 0; k < K; ++k) xrow[k] = 0.0f;
+        for (int64_t g = 0; g < K / 4; ++g) {
+            unsigned nib = (meta_canon[m * (K / 16) + g / 4] >> (4 * (g % 4))) & 0xfu;
+            xrow[4 * g + (nib & 3u)] = oracle_e4m3_decode(values_q[m * (K / 2) + 2 * g + 0]);
+            xrow[4 * g + (nib >> 2)] = oracle_e4m3_decode(values_q[m * (K / 2) + 2 * g + 1]);
+        }
+        for (int64_t n = 0; n < N; ++n) {
+            float a = 0.0f;
+            for (int64_t k = 0; k < K; ++k) a += xrow[k] * oracle_e4m3_decode(Wq[n * K + k]);
+            acc[i * N + n] = a;
+        }
+        free(xrow);
+    }
+}
+
+/* Whole FP8 path for a set of rows.  comp_mode: 0 none, 1 per-row norm compensation.
+ * row_scale_out[m] = s_m * act_scale_m (what the epilogue multiplies row m by). */
+ORACLE_API void oracle_act_sparse_linear_fp8(const uint16_t* X, int64_t M, int64_t K, int64_t ldx,
+                                             const uint8_t* Wq, const float* wscale, int64_t N,
+                                             const uint16_t* bias, int comp_mode, const uint16_t* Yr, int64_t ldr,
+                                             const int64_t* rows, int64_t n_rows, uint8_t* values_q,
+                                             uint16_t* meta_canon, float* row_scale_out, float* acc_scratch,
+                                             float* Y) {
+    float* act = (float*)malloc((size_t)M * sizeof(float));
+    float* s = (float*)malloc((size_t)M * sizeof(float));
+    oracle_compress_fp8(X, M, K, ldx, values_q, meta_canon, act);
+    oracle_row_scale(X, M, K, ldx, comp_mode == 1 ? 1 : 0, s);
+    for (int64_t m = 0; m < M; ++m) row_scale_out[m] = s[m] * act[m];
+    oracle_gemm_fp8_f32(values_q, meta_canon, M, K, Wq, N, rows, n_rows, acc_scratch);
+    if (!rows) n_rows = M;
+    for (int64_t i = 0; i < n_rows; ++i) {
+        const int64_t m = rows ? rows[i] : i;
+        for (int64_t n = 0; n < N; ++n) {
+            float y = row_scale_out[m] * wscale[n] * acc_scratch[i * N + n];
+            if (bias) y = y + bf16_to_f32(bias[n]);
+            if (Yr) y = y + bf16_to_f32(Yr[m * ldr + n]);
+            Y[i * N + n] = y;
+        }
+    }
+    free(act);
+    free(s);
 }

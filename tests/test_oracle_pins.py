@@ -407,6 +407,101 @@ def test_group_mode_whole_path_is_the_product_of_the_scaled_sparse_activation():
     assert (out["scale"] == 1.0).all()
 
 
+# --------------------------------------------------------------------------- FP8 composition ---
+
+def test_e4m3_codec_matches_the_library_conversion_and_saturates():
+    # decode: all 256 codes against torch's float8_e4m3fn
+    codes = torch.arange(256, dtype=torch.uint8)
+    ref = codes.view(torch.float8_e4m3fn).float().numpy()
+    got = oracle.e4m3_decode(codes.numpy())
+    assert (np.isnan(got) == np.isnan(ref)).all() and (got[~np.isnan(ref)] == ref[~np.isnan(ref)]).all()
+    # encode: random values, every grid point, every midpoint (ties to even), inside the finite range
+    g = torch.Generator().manual_seed(31)
+    finite = np.sort(ref[~np.isnan(ref) & (ref >= 0)])
+    mids = (finite[1:] + finite[:-1]) / 2
+    x = np.concatenate([finite, mids, np.nextafter(mids, 0).astype(np.float32), np.nextafter(mids, 1e9).astype(np.float32),
+                        (torch.randn(20000, generator=g) * torch.exp(2 * torch.randn(20000, generator=g))).numpy()])
+    x = np.concatenate([x, -x]).astype(np.float32)
+    x = x[np.abs(x) <= 464.0]
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert (oracle.e4m3_encode(x) == want).all()
+    # satfinite: beyond the range, and Inf, give +-448; NaN stays NaN
+    big = oracle.e4m3_encode(np.array([464.0, 465.0, 1e6, np.inf, -500.0, -np.inf], dtype=np.float32))
+    assert (big == np.array([0x7E, 0x7E, 0x7E, 0x7E, 0xFE, 0xFE], dtype=np.uint8)).all()
+    assert np.isnan(oracle.e4m3_decode(oracle.e4m3_encode(np.array([np.nan], dtype=np.float32)))).all()
+
+
+def test_fp8_activation_codes_closed_forms():
+    """Row amax maps to +-448 exactly; a row of zeros gives zero codes and a zero scale; the mask
+    is the bf16 one; the decoded codes times the scale reproduce the kept values to E4M3 accuracy."""
+    g = torch.Generator().manual_seed(32)
+    M, K = 24, 256
+    x = torch.randn(M, K, generator=g)
+    x[3] = 0.0
+    x[5, 17] = 100.0
+    x = x.to(torch.bfloat16)
+    X = inputs.as_u16(x)
+    vq, meta, sc = oracle.compress_fp8(X)
+    v0, meta0 = oracle.compress(X)
+    assert (meta == meta0).all()
+    dec = oracle.e4m3_decode(vq)
+    amax = x.float().abs().max(dim=1).values.numpy()
+    assert (np.abs(dec).max(axis=1)[amax > 0] == 448.0).all()
+    assert sc[3] == 0.0 and (vq[3] == 0).all()
+    np.testing.assert_allclose(sc, amax / 448.0, rtol=1e-6)
+    kept = inputs.from_u16(v0).float().numpy()
+    err = np.abs(dec * sc[:, None] - kept)
+    # E4M3: 3 mantissa bits -> half a step is 2^-4 relative for normals; below 2^-6 of the row's
+    # maximum / 448 * ... the grid is absolute (subnormals): 2^-10 * scale
+    assert (err <= np.maximum(np.abs(kept) * 2.0 ** -4, sc[:, None] * 2.0 ** -10) * 1.0001).all()
+
+
+def test_fp8_weight_quantisation_modes():
+    g = torch.Generator().manual_seed(33)
+    N, K = 12, 64
+    w = (torch.randn(N, K, generator=g) * 0.05).to(torch.bfloat16)
+    Wq, ws = oracle.quantize_weights_fp8(inputs.as_u16(w), per_channel=False)
+    assert (ws == 1.0).all()
+    assert (Wq == w.float().to(torch.float8_e4m3fn).view(torch.uint8).numpy()).all()   # a direct cast
+    Wq, ws = oracle.quantize_weights_fp8(inputs.as_u16(w), per_channel=True)
+    amax = w.float().abs().max(dim=1).values.numpy()
+    np.testing.assert_allclose(ws, amax / 448.0, rtol=1e-6)
+    assert (np.abs(oracle.e4m3_decode(Wq)).max(axis=1) == 448.0).all()
+
+
+def test_fp8_whole_path_is_the_product_of_the_dequantised_operands():
+    g = torch.Generator().manual_seed(34)
+    M, K, N = 16, 256, 24
+    x = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    w = (torch.randn(N, K, generator=g) * K ** -0.5).to(torch.bfloat16)
+    b = (torch.randn(N, generator=g) * 0.1).to(torch.bfloat16)
+    X = inputs.as_u16(x)
+    for per_channel in (False, True):
+        Wq, ws = oracle.quantize_weights_fp8(inputs.as_u16(w), per_channel)
+        for mode in (oracle.COMP_NONE, oracle.COMP_ROW):
+            out = oracle.act_sparse_linear_fp8(X, Wq, ws, bias=inputs.as_u16(b), comp_mode=mode)
+            vq, meta, sc = oracle.compress_fp8(X)
+            assert (out["values_q"] == vq).all() and (out["meta_canon"] == meta).all()
+            # restated: scatter the decoded codes by the metadata, multiply in fp64
+            xs = np.zeros((M, K))
+            dec = oracle.e4m3_decode(vq).astype(np.float64).reshape(M, K // 4, 2)
+            for m in range(M):
+                for gi in range(K // 4):
+                    nib = (int(meta[m, gi // 4]) >> (4 * (gi % 4))) & 0xF
+                    xs[m, 4 * gi + (nib & 3)] = dec[m, gi, 0]
+                    xs[m, 4 * gi + (nib >> 2)] = dec[m, gi, 1]
+            s = oracle.row_scale(X, mode).astype(np.float64) * sc.astype(np.float64)
+            ref = (xs @ oracle.e4m3_decode(Wq).astype(np.float64).T) * s[:, None] * ws.astype(np.float64)[None, :] \
+                + b.double().numpy()[None, :]
+            np.testing.assert_allclose(out["Y"], ref, rtol=1e-4, atol=1e-5)
+            np.testing.assert_allclose(out["row_scale"], s, rtol=1e-6)
+            # and the FP8 layer stays close to the bf16 sparse layer it approximates
+            # (per-channel weight scales only: a direct cast of weights this small sits in E4M3's subnormals)
+            if per_channel:
+                y16 = oracle.act_sparse_linear(X, inputs.as_u16(w), bias=inputs.as_u16(b), comp_mode=mode)["Y"]
+                assert np.linalg.norm(out["Y"] - y16) / np.linalg.norm(y16) < 0.06
+
+
 def test_lora_rows_subset_equals_full_rows():
     g = torch.Generator().manual_seed(12)
     M, K, R, N = 20, 128, 8, 24
