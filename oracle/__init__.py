@@ -280,6 +280,13 @@ def compress_fp8(X):
     return vq, meta, sc
 
 
+def meta_canon_to_hw_fp8(meta_canon, M: int, K: int) -> np.ndarray:
+    meta_canon = _u16(meta_canon, "meta_canon")
+    out = np.empty(((M + 127) // 128) * (K // 128) * 2048, dtype=np.uint8)
+    _load().oracle_meta_canon_to_hw_fp8(_p(meta_canon), _i64(M), _i64(K), _p(out))
+    return out
+
+
 def act_sparse_linear_fp8(X, Wq, wscale, bias=None, comp_mode=COMP_NONE, Yr=None, rows=None):
     """Whole FP8 path.  -> dict(values_q, meta_canon, row_scale (= s * act_scale), Y[fp32, rows x N])."""
     X, M, K = _check_x(X)

@@ -406,7 +406,10 @@ ORACLE_API void oracle_act_sparse_linear(const uint16_t* X, int64_t M, int64_t K
  * The paper fixes neither the granularity of the activation scale nor any rounding; the
  * reading taken (and restated in the CUDA library's header) is:
  *   selection      on the bf16 activations, as everywhere else (the mask does not change);
- *   activation     per token row m: amax_m = max |x~| over the kept values (= max over the row),
+ *   activation     per token row m: amax_m = the largest magnitude of the row in the order the
+ *                  selection uses (the 15 non-sign bits as an integer: NaN > Inf > finite), so it
+ *                  is also the largest kept magnitude, and a NaN in the row makes the row's
+ *                  scale NaN (it propagates to Y as in a dense layer),
  *                  inv_m = 448 / amax_m (fp32 division; 0 if amax_m = 0),
  *                  code = e4m3_rne_satfinite(x~ * inv_m)  (fp32 product, then one rounding),
  *                  act_scale_m = amax_m / 448 (fp32 division);
@@ -463,18 +466,35 @@ ORACLE_API void oracle_e4m3_encode_array(const float* in, int64_t n, uint8_t* ou
     for (int64_t i = 0; i < n; ++i) out[i] = oracle_e4m3_encode(in[i]);
 }
 
+/* Metadata order of the FP8 (kind f8f6f4) sparse MMA: one instruction covers 64 logical K and
+ * reads, for row r of its 128 rows, 64 metadata bits from tensor-memory lane r in natural order
+ * (nibble of group g in bits 4g..4g+3).  Stored as blocks of 128 rows x 128 K-elements, 2048 bytes
+ * each, block (rb, kb) at byte (rb * K/128 + kb) * 2048; inside a block byte = r * 16 + g / 2 with
+ * r = row in block, g = (k % 128) / 4, group g in bits 4 * (g % 2) of that byte.  Rows past M in
+ * the last block carry the legal pattern 0x4. */
+ORACLE_API void oracle_meta_canon_to_hw_fp8(const uint16_t* meta_canon, int64_t M, int64_t K, uint8_t* meta_hw) {
+    const int64_t RB = (M + 127) / 128, KB = K / 128;
+    memset(meta_hw, 0x44, (size_t)(RB * KB * 2048));
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t g = 0; g < K / 4; ++g) {
+            const unsigned nib = (meta_canon[m * (K / 16) + g / 4] >> (4 * (g % 4))) & 0xfu;
+            const int64_t rb = m / 128, r = m % 128, kb = (4 * g) / 128, gl = g % 32;
+            uint8_t* byte = meta_hw + (rb * KB + kb) * 2048 + r * 16 + gl / 2;
+            *byte = (uint8_t)((*byte & ~(0xfu << (4 * (gl % 2)))) | (nib << (4 * (gl % 2))));
+        }
+}
+
 /* Weights: mode 0 direct cast, 1 symmetric per output channel.  Wq is N x K codes, wscale N floats. */
 ORACLE_API void oracle_quantize_weights_fp8(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode,
                                             uint8_t* Wq, float* wscale) {
     for (int64_t n = 0; n < N; ++n) {
         float inv = 1.0f, sc = 1.0f;
         if (mode == 1) {
-            float amax = 0.0f;
-            for (int64_t k = 0; k < K; ++k) {
-                float a = fabsf(bf16_to_f32(W[n * ldw + k]));
-                if (a > amax) amax = a;                        /* NaN never raises the maximum */
-            }
-            inv = amax > 0.0f ? 448.0f / amax : 0.0f;
+            unsigned top = 0;
+            for (int64_t k = 0; k < K; ++k)
+                if (mag15(W[n * ldw + k]) > top) top = mag15(W[n * ldw + k]);
+            const float amax = bf16_to_f32((uint16_t)top);
+            inv = amax > 0.0f ? 448.0f / amax : 0.0f;          /* 0 for amax = 0 and for NaN */
             sc = amax / 448.0f;
         }
         for (int64_t k = 0; k < K; ++k) Wq[n * K + k] = oracle_e4m3_encode(bf16_to_f32(W[n * ldw + k]) * inv);
@@ -489,12 +509,11 @@ ORACLE_API void oracle_compress_fp8(const uint16_t* X, int64_t M, int64_t K, int
     const int64_t G = K / 4;
     memset(meta_canon, 0, (size_t)(M * (K / 16)) * sizeof(uint16_t));
     for (int64_t m = 0; m < M; ++m) {
-        float amax = 0.0f;
-        for (int64_t k = 0; k < K; ++k) {
-            float a = fabsf(bf16_to_f32(X[m * ldx + k]));
-            if (a > amax) amax = a;
-        }
-        const float inv = amax > 0.0f ? 448.0f / amax : 0.0f;
+        unsigned top = 0;
+        for (int64_t k = 0; k < K; ++k)
+            if (mag15(X[m * ldx + k]) > top) top = mag15(X[m * ldx + k]);
+        const float amax = bf16_to_f32((uint16_t)top);
+        const float inv = amax > 0.0f ? 448.0f / amax : 0.0f;  /* 0 for amax = 0 and for NaN */
         act_scale[m] = amax / 448.0f;
         for (int64_t g = 0; g < G; ++g) {
             const uint16_t* grp = X + m * ldx + 4 * g;

@@ -456,6 +456,21 @@ def test_fp8_activation_codes_closed_forms():
     assert (err <= np.maximum(np.abs(kept) * 2.0 ** -4, sc[:, None] * 2.0 ** -10) * 1.0001).all()
 
 
+def test_fp8_metadata_order_is_the_rows_bytes_block_by_block():
+    """Independent restatement: per (128-row, 128-K) block, row r's 16 bytes are the row's 8
+    canonical little-endian words of that K block; rows past M are 0x44."""
+    g = torch.Generator().manual_seed(35)
+    M, K = 200, 384
+    X = inputs.as_u16(torch.randn(M, K, generator=g).to(torch.bfloat16))
+    _, meta = oracle.compress(X)
+    hw = oracle.meta_canon_to_hw_fp8(meta, M, K).reshape(2, 3, 128, 16)
+    rows = meta.view(np.uint8).reshape(M, K // 128, 16)          # little-endian host
+    for rb in range(2):
+        n = min(128, M - rb * 128)
+        assert (hw[rb, :, :n, :] == rows[rb * 128: rb * 128 + n].transpose(1, 0, 2)).all()
+        assert (hw[rb, :, n:, :] == 0x44).all()
+
+
 def test_fp8_weight_quantisation_modes():
     g = torch.Generator().manual_seed(33)
     N, K = 12, 64
