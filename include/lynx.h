@@ -241,6 +241,47 @@ LYNX_API lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, i
                                                  lynx_comp_mode mode, const void* residual,
                                                  int64_t ldr, void* Y, int64_t ldy, void* stream);
 
+/* ---- FP8 composition (the paper's W8A8 compatibility experiment: symmetric FP8 quantisation of
+ *      the activations, weights cast to FP8; 2:4 is one of the sparse tensor core's FP8 formats) ----
+ * FP8 = E4M3 (1-4-3 bits, bias 7, no infinities, largest finite 448).  The paper fixes neither the
+ * granularity of the activation scale nor the rounding; this library's rules, all in fp32 with
+ * IEEE operations:
+ *   selection   on the bf16 activations exactly as in lynx_prune_compress (same mask, same nibbles);
+ *   activation  per token row m: amax_m = the row's largest magnitude in the selection's order
+ *               (15 non-sign bits as an integer, so NaN > Inf > finite), inv_m = amax_m > 0 ?
+ *               448 / amax_m : 0, code = e4m3(x * inv_m) rounded to nearest even, finite overflow
+ *               saturating to +-448; act_scale_m = amax_m / 448;
+ *   weights     per_channel = 0: code = e4m3(w) (a direct cast), wscale[n] = 1;
+ *               per_channel = 1: the same symmetric rule per output channel n;
+ *   product     fp32 accumulation on the sparse tensor cores (kind f8f6f4, K = 64 per instruction);
+ *   epilogue    Y = bf16_rne( row_scale[m] * wscale[n] * acc + bias[n] + Y_r[m,n] ) with
+ *               row_scale[m] = s_m * act_scale_m, s_m the per-row norm compensation of the bf16
+ *               row (LYNX_COMP_ROW) or 1 (LYNX_COMP_NONE).
+ * Layouts: values_q is M x K/2 bytes row-major; Wq is N x K bytes row-major, leading dimension
+ * ldwq bytes (multiple of 16); wscale [N] fp32 (NULL = all 1).  K % 256 == 0.  meta has the size
+ * lynx_meta_bytes(M, K) but its own order: blocks of 128 rows x 128 K-elements, 2048 bytes each,
+ * block (rb, kb) at byte (rb * K/128 + kb) * 2048, inside a block row r's 16 bytes at r * 16 with
+ * group g = (k % 128) / 4 in bits 4 * (g % 2) of byte g / 2; rows past M hold 0x4 nibbles.
+ * lynx_prune_compress_fp8 reads X twice (row maxima first; the second pass normally hits the L2)
+ * and needs no scratch.  The low-rank branch, LYNX_COMP_TENSOR / GROUP and the one-kernel mode are
+ * not available in FP8.
+ */
+LYNX_API lynx_status lynx_quantize_weights_fp8(lynx_ctx* ctx, const void* W, int64_t N, int64_t K,
+                                               int64_t ldw, int per_channel, void* Wq, float* wscale,
+                                               void* stream);
+LYNX_API lynx_status lynx_prune_compress_fp8(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
+                                             int64_t ldx, void* values_q, void* meta,
+                                             float* row_scale, lynx_comp_mode mode, void* stream);
+LYNX_API lynx_status lynx_sparse_linear_fp8(lynx_ctx* ctx, const void* values_q, const void* meta,
+                                            int64_t M, int64_t K, const void* Wq, int64_t N,
+                                            int64_t ldwq, const float* wscale, const void* bias,
+                                            const lynx_comp* comp, void* Y, int64_t ldy, void* stream);
+LYNX_API lynx_status lynx_act_sparse_linear_fp8(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
+                                                int64_t ldx, const void* Wq, int64_t N, int64_t ldwq,
+                                                const float* wscale, const void* bias,
+                                                lynx_comp_mode mode, const void* residual, int64_t ldr,
+                                                void* Y, int64_t ldy, void* stream);
+
 /* ---- inspection helpers ------------------------------------------------------------------------ */
 
 /* Hardware-order metadata -> canonical form: uint16 [M x K/16], nibble (g%4) of group g in bits

@@ -23,6 +23,8 @@ EXPORTS = [
     "lynx_sparse_linear", "lynx_act_sparse_linear", "lynx_act_sparse_linear_host",
     "lynx_meta_to_canonical", "lynx_decompress", "lynx_launch_count", "lynx_prune_compress_static",
     "lynx_reserve_lora", "lynx_lora_down", "lynx_sparse_linear_lora", "lynx_act_sparse_linear_lora",
+    "lynx_quantize_weights_fp8", "lynx_prune_compress_fp8", "lynx_sparse_linear_fp8",
+    "lynx_act_sparse_linear_fp8",
 ]
 
 
@@ -79,6 +81,12 @@ def load_library() -> ctypes.CDLL:
                                             i64, vp, i64, i64, vp, i64, vp]
     lib.lynx_act_sparse_linear_lora.argtypes = [vp, vp, i64, i64, i64, vp, i64, i64, vp, vp, i64, vp, i64, i64,
                                                 i32, vp, i64, vp, i64, vp]
+    lib.lynx_quantize_weights_fp8.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
+    lib.lynx_prune_compress_fp8.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, i32, vp]
+    lib.lynx_sparse_linear_fp8.argtypes = [vp, vp, vp, i64, i64, vp, i64, i64, vp, vp, ctypes.POINTER(_Comp), vp,
+                                           i64, vp]
+    lib.lynx_act_sparse_linear_fp8.argtypes = [vp, vp, i64, i64, i64, vp, i64, i64, vp, vp, i32, vp, i64, vp, i64,
+                                               vp]
     lib.lynx_launch_count.argtypes = [vp]
     lib.lynx_launch_count.restype = i64
     _lib = lib
@@ -283,6 +291,58 @@ class Lynx:
                                                      mode, _ptr(residual),
                                                      0 if residual is None else residual.stride(0), _ptr(out),
                                                      out.stride(0), _stream()), "lynx_act_sparse_linear_lora")
+        return out
+
+    # -- FP8 composition -----------------------------------------------------------------------
+    def quantize_weights_fp8(self, W: torch.Tensor, per_channel: bool = True):
+        """-> (Wq uint8 [N, K] E4M3 codes, wscale float32 [N])"""
+        _bf16_2d(W, "W")
+        N, K = W.shape
+        Wq = torch.empty((N, K), dtype=torch.uint8, device=W.device)
+        ws = torch.empty(N, dtype=torch.float32, device=W.device)
+        _check(self._lib.lynx_quantize_weights_fp8(self._h, _ptr(W), N, K, W.stride(0), 1 if per_channel else 0,
+                                                   _ptr(Wq), _ptr(ws), _stream()), "lynx_quantize_weights_fp8")
+        return Wq, ws
+
+    def prune_compress_fp8(self, X: torch.Tensor, mode: int = COMP_NONE, values_q=None, meta=None, row_scale=None):
+        """-> (values_q uint8 [M, K/2], meta uint8, row_scale float32 [M] = s * amax / 448)"""
+        _bf16_2d(X, "X")
+        M, K = X.shape
+        if values_q is None:
+            values_q = torch.empty((M, K // 2), dtype=torch.uint8, device=X.device)
+        if meta is None:
+            meta = torch.empty(meta_bytes(M, K), dtype=torch.uint8, device=X.device)
+        if row_scale is None:
+            row_scale = torch.empty(M, dtype=torch.float32, device=X.device)
+        _check(self._lib.lynx_prune_compress_fp8(self._h, _ptr(X), M, K, X.stride(0), _ptr(values_q), _ptr(meta),
+                                                 _ptr(row_scale), mode, _stream()), "lynx_prune_compress_fp8")
+        return values_q, meta, row_scale
+
+    def sparse_linear_fp8(self, values_q: torch.Tensor, meta: torch.Tensor, Wq: torch.Tensor, wscale=None,
+                          bias=None, row_scale=None, residual=None, out=None) -> torch.Tensor:
+        M, K = values_q.shape[0], values_q.shape[1] * 2
+        N = Wq.shape[0]
+        if out is None:
+            out = torch.empty((M, N), dtype=torch.bfloat16, device=values_q.device)
+        comp = _Comp(None if row_scale is None else row_scale.data_ptr(),
+                     None if residual is None else residual.data_ptr(),
+                     0 if residual is None else residual.stride(0))
+        _check(self._lib.lynx_sparse_linear_fp8(self._h, _ptr(values_q), _ptr(meta), M, K, _ptr(Wq), N, Wq.stride(0),
+                                                _ptr(wscale), _ptr(bias), ctypes.byref(comp), _ptr(out),
+                                                out.stride(0), _stream()), "lynx_sparse_linear_fp8")
+        return out
+
+    def act_sparse_linear_fp8(self, X: torch.Tensor, Wq: torch.Tensor, wscale=None, bias=None,
+                              mode: int = COMP_NONE, residual=None, out=None) -> torch.Tensor:
+        _bf16_2d(X, "X")
+        M, K = X.shape
+        N = Wq.shape[0]
+        if out is None:
+            out = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+        _check(self._lib.lynx_act_sparse_linear_fp8(self._h, _ptr(X), M, K, X.stride(0), _ptr(Wq), N, Wq.stride(0),
+                                                    _ptr(wscale), _ptr(bias), mode, _ptr(residual),
+                                                    0 if residual is None else residual.stride(0), _ptr(out),
+                                                    out.stride(0), _stream()), "lynx_act_sparse_linear_fp8")
         return out
 
     # -- inspection ----------------------------------------------------------------------------

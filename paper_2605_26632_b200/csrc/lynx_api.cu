@@ -14,6 +14,7 @@
 #include "sparse_gemm.cuh"
 #include "fused_linear.cuh"
 #include "lora_down.cuh"
+#include "fp8_path.cuh"
 
 using namespace lynx;
 
@@ -232,6 +233,7 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     p.row_scale = comp ? comp->row_scale : nullptr;
     p.scale_partial = ss ? ss->partial : nullptr;
     p.scale_ks = ss ? ss->ks : 0;
+    p.col_scale = nullptr;
     p.bias = static_cast<const uint16_t*>(bias);
     p.residual = comp ? static_cast<const uint16_t*>(comp->residual) : nullptr;
     p.ldr = comp ? comp->ldr : 0;
@@ -330,9 +332,8 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
 // Model: rounds of tiles over the CTA pairs x (K blocks x measured time per K block + exposed
 // epilogue).  Per-K-block times (us) are measured B200 figures for each tile shape; the 256-wide
 // tile has one accumulator buffer, so its epilogue is not hidden.
-int pick_gemm_cfg(const lynx_ctx* ctx, int64_t M, int64_t N, int64_t K, int lora_steps) {
-    if (ctx->gemm_cfg != 0) return ctx->gemm_cfg;
-    const int pairs = ctx->num_sms / 2;
+int pick_gemm_cfg_model(int num_sms, int64_t M, int64_t N, int64_t K, int lora_steps) {
+    const int pairs = num_sms / 2;
     const double kb = (double)(K / 128) + lora_steps;
     struct { int id, bn; double t_kb, epi; } cand[4] = {
         {7, 240, 0.465, 0.6}, {5, 256, 0.50, 3.0}, {4, 192, 0.415, 0.6}, {6, 128, 0.345, 0.5}};
@@ -345,6 +346,10 @@ int pick_gemm_cfg(const lynx_ctx* ctx, int64_t M, int64_t N, int64_t K, int lora
         if (t < best) { best = t; cfg = c.id; }
     }
     return cfg;
+}
+int pick_gemm_cfg(const lynx_ctx* ctx, int64_t M, int64_t N, int64_t K, int lora_steps) {
+    if (ctx->gemm_cfg != 0) return ctx->gemm_cfg;
+    return pick_gemm_cfg_model(ctx->num_sms, M, N, K, lora_steps);
 }
 // every tile but the 2-CTA 256 x 128 one has room in its W slot for a phase-0 stage
 bool cfg_supports_l0(int cfg) { return cfg >= 1 && cfg <= 7 && cfg != 6; }
@@ -365,6 +370,82 @@ lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int
         default: return LYNX_ERR_INVALID_ARG;
     }
 #undef LYNX_GEMM_ARGS
+}
+
+// FP8 (E4M3) instantiation: byte tensor maps, K blocks of 256, optional per-channel weight scale.
+template <class Cfg>
+lynx_status launch_gemm_fp8_cfg(lynx_ctx* ctx, const void* values_q, const void* meta, int64_t M, int64_t K,
+                                const void* Wq, int64_t N, int64_t ldwq, const float* wscale, const void* bias,
+                                const lynx_comp* comp, void* Y, int64_t ldy, cudaStream_t st) {
+    static_assert(Cfg::FP8, "FP8 configuration expected");
+    CUtensorMap ta, tb, te, ty;
+    const uint64_t rb = (uint64_t)((M + 127) / 128), kb128 = (uint64_t)(K / 128);
+    if (!make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, values_q, (uint64_t)M, (uint64_t)(K / 2),
+                      (uint64_t)(K / 2), 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldwq, 128,
+                      Cfg::BN_CTA, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&te, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, meta, rb * kb128 * 2, 256, 1024, 256,
+                      Cfg::E_BYTES / 1024, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, Cfg::CH,
+                      32, Cfg::CH == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE))
+        return LYNX_ERR_CUDA;
+    GemmParams p = {};
+    p.M = M; p.N = N; p.K = K;
+    p.row_scale = comp ? comp->row_scale : nullptr;
+    p.col_scale = wscale;
+    p.bias = static_cast<const uint16_t*>(bias);
+    p.residual = comp ? static_cast<const uint16_t*>(comp->residual) : nullptr;
+    p.ldr = comp ? comp->ldr : 0;
+    p.dev_error = ctx->err_dev;
+    p.tiles_m = (int)((M + Cfg::BM * Cfg::CG - 1) / (Cfg::BM * Cfg::CG));
+    p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
+    p.l0_splits = 1;
+    auto kern = sparse_gemm_kernel<Cfg, false>;
+    static bool attr_set = false;  // per instantiation
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
+            return LYNX_ERR_CUDA;
+        attr_set = true;
+    }
+    const int tiles = p.tiles_m * p.tiles_n;
+    int clusters = ctx->num_sms / Cfg::CG;
+    if (clusters > tiles) clusters = tiles;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(clusters * Cfg::CG));
+    cfg.blockDim = dim3(Cfg::THREADS);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = Cfg::CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, kern, ta, tb, te, ty, ta, tb, ta, tb, p) != cudaSuccess) return LYNX_ERR_CUDA;
+    ctx->launches++;
+    return LYNX_OK;
+}
+
+// FP8 tile choice: the development override if it names a CTA-pair tile, else the cost model's
+// choice among the same pair tiles (a stage is 256 K here; relative times as for bf16).
+lynx_status launch_gemm_fp8(lynx_ctx* ctx, const void* values_q, const void* meta, int64_t M, int64_t K,
+                            const void* Wq, int64_t N, int64_t ldwq, const float* wscale, const void* bias,
+                            const lynx_comp* comp, void* Y, int64_t ldy, cudaStream_t st) {
+    int cfg = ctx->gemm_cfg;
+    if (cfg != 4 && cfg != 6 && cfg != 7) {
+        cfg = pick_gemm_cfg_model(ctx->num_sms, M, N, K / 2, 0);
+        if (cfg == 5) cfg = 7;  // the 256-wide tile has no FP8 instantiation (no tensor memory left for metadata)
+    }
+#define LYNX_FP8_ARGS ctx, values_q, meta, M, K, Wq, N, ldwq, wscale, bias, comp, Y, ldy, st
+    switch (cfg) {
+        case 4: return launch_gemm_fp8_cfg<GemmCfg<192, 2, 4, 2, true>>(LYNX_FP8_ARGS);
+        case 6: return launch_gemm_fp8_cfg<GemmCfg<128, 2, 5, 2, true>>(LYNX_FP8_ARGS);
+        default: return launch_gemm_fp8_cfg<GemmCfg<240, 2, 4, 2, true>>(LYNX_FP8_ARGS);
+    }
+#undef LYNX_FP8_ARGS
 }
 
 // One-kernel path: raw X is pruned inside the GEMM kernel.
@@ -922,6 +1003,109 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
     s = lynx_lora_down(ctx, X, M, K, ldx, LB, R, ldlb, scale, T, R, stream);
     if (s != LYNX_OK) return s;
     return lynx_sparse_linear_lora(ctx, values, meta, M, K, W, N, ldw, bias, &comp, T, R, LA, R, ldla, Y, ldy, stream);
+}
+
+// ------------------------------------------------------------------------- FP8 composition ------
+
+static lynx_status check_fp8_shape(lynx_ctx* ctx, int64_t M, int64_t K) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if (K % 256 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    return LYNX_OK;
+}
+
+lynx_status lynx_quantize_weights_fp8(lynx_ctx* ctx, const void* W, int64_t N, int64_t K, int64_t ldw,
+                                      int per_channel, void* Wq, float* wscale, void* stream) {
+    if (!ctx || !W || !Wq || !wscale || N < 1 || K < 2) return LYNX_ERR_INVALID_ARG;
+    if (K % 2 != 0 || ldw < K) return LYNX_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(Wq) & 1u) return LYNX_ERR_ALIGNMENT;
+    quantize_weights_fp8_kernel<<<(unsigned)N, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint16_t*>(W), N, K, ldw, per_channel ? 1 : 0, static_cast<uint8_t*>(Wq), wscale);
+    ctx->launches++;
+    return cuda_ok(cudaGetLastError());
+}
+
+lynx_status lynx_prune_compress_fp8(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, void* values_q,
+                                    void* meta, float* row_scale, lynx_comp_mode mode, void* stream) {
+    lynx_status s = check_fp8_shape(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if (!X || !values_q || !meta || !row_scale) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW) return LYNX_ERR_INVALID_ARG;
+    if (ldx < K) return LYNX_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(X) & 31u) || !aligned16(values_q) || !aligned16(meta) || (ldx % 16) != 0)
+        return LYNX_ERR_ALIGNMENT;
+    if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+    cudaLaunchConfig_t pc = {};
+    pc.gridDim = dim3((unsigned)(((M + 127) / 128) * 8));
+    pc.blockDim = dim3(FP8_PRUNE_WARPS * 32);
+    pc.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute pa[1];
+    pa[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pa[0].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
+    pc.attrs = pa;
+    pc.numAttrs = 1;
+    const uint16_t* Xp = static_cast<const uint16_t*>(X);
+    uint8_t* vp = static_cast<uint8_t*>(values_q);
+    uint8_t* mp = static_cast<uint8_t*>(meta);
+    cudaError_t e = (mode == LYNX_COMP_ROW)
+                        ? cudaLaunchKernelEx(&pc, prune_compress_fp8_kernel<true>, Xp, M, K, ldx, vp, mp, row_scale)
+                        : cudaLaunchKernelEx(&pc, prune_compress_fp8_kernel<false>, Xp, M, K, ldx, vp, mp, row_scale);
+    if (e != cudaSuccess) return LYNX_ERR_CUDA;
+    ctx->launches++;
+    return LYNX_OK;
+}
+
+lynx_status lynx_sparse_linear_fp8(lynx_ctx* ctx, const void* values_q, const void* meta, int64_t M, int64_t K,
+                                   const void* Wq, int64_t N, int64_t ldwq, const float* wscale, const void* bias,
+                                   const lynx_comp* comp, void* Y, int64_t ldy, void* stream) {
+    lynx_status s = check_fp8_shape(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if (!values_q || !meta || !Wq || !Y || N < 8) return LYNX_ERR_INVALID_ARG;
+    if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    if (ldwq < K || ldy < N) return LYNX_ERR_INVALID_ARG;
+    if (!aligned16(values_q) || !aligned16(meta) || !aligned16(Wq) || !aligned16(Y) || (ldwq % 16) || (ldy % 8))
+        return LYNX_ERR_ALIGNMENT;
+    if ((bias && !aligned16(bias)) || (wscale && !aligned16(wscale))) return LYNX_ERR_ALIGNMENT;
+    if (comp && comp->residual) {
+        if (comp->ldr < N) return LYNX_ERR_INVALID_ARG;
+        if (!aligned16(comp->residual) || (comp->ldr % 8)) return LYNX_ERR_ALIGNMENT;
+    }
+    if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+    return launch_gemm_fp8(ctx, values_q, meta, M, K, Wq, N, ldwq, wscale, bias, comp, Y, ldy,
+                           static_cast<cudaStream_t>(stream));
+}
+
+lynx_status lynx_act_sparse_linear_fp8(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx,
+                                       const void* Wq, int64_t N, int64_t ldwq, const float* wscale,
+                                       const void* bias, lynx_comp_mode mode, const void* residual, int64_t ldr,
+                                       void* Y, int64_t ldy, void* stream) {
+    lynx_status s = check_fp8_shape(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    // every argument is checked before the first launch
+    if (!X || !Wq || !Y || N < 8) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW) return LYNX_ERR_INVALID_ARG;
+    if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
+    if (ldx < K || ldwq < K || ldy < N || (residual && ldr < N)) return LYNX_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(X) & 31u) || (ldx % 16) || !aligned16(Wq) || !aligned16(Y) || (ldwq % 16) ||
+        (ldy % 8) || (bias && !aligned16(bias)) || (wscale && !aligned16(wscale)) ||
+        (residual && (!aligned16(residual) || (ldr % 8))))
+        return LYNX_ERR_ALIGNMENT;
+    ScratchLayout L = scratch_layout(M, N, K);
+    {
+        std::lock_guard<std::mutex> lock(ctx->mu);
+        if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
+    }
+    char* base = static_cast<char*>(ctx->scratch);
+    void* values_q = base + L.values;  // (sized for bf16 values: twice what the codes need)
+    void* meta = base + L.meta;
+    float* scale = reinterpret_cast<float*>(base + L.scale);
+    s = lynx_prune_compress_fp8(ctx, X, M, K, ldx, values_q, meta, scale, mode, stream);
+    if (s != LYNX_OK) return s;
+    lynx_comp comp;
+    comp.row_scale = scale;
+    comp.residual = residual;
+    comp.ldr = ldr;
+    return lynx_sparse_linear_fp8(ctx, values_q, meta, M, K, Wq, N, ldwq, wscale, bias, &comp, Y, ldy, stream);
 }
 
 lynx_status lynx_meta_to_canonical(lynx_ctx* ctx, const void* meta, int64_t M, int64_t K, void* meta_canon,

@@ -329,6 +329,27 @@ __device__ __forceinline__ void mma_bf16_lh(uint32_t d_tmem, uint32_t a_lo, uint
             : "memory");
 }
 
+// FP8 (E4M3 x E4M3 -> fp32) sparse form: K = 64 logical per instruction, metadata in two
+// consecutive tensor-memory columns per lane in natural order.
+template <int CG>
+__device__ __forceinline__ void mma_sp_f8_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                             uint32_t e_tmem, uint32_t idesc, uint32_t accumulate) {
+    if constexpr (CG == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.sp.cta_group::1.kind::f8f6f4 [%0], da, db, [%4], %5, p;\n\t}" ::"r"(d_tmem),
+            "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(e_tmem), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.sp.cta_group::2.kind::f8f6f4 [%0], da, db, [%4], %5, p;\n\t}" ::"r"(d_tmem),
+            "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(e_tmem), "r"(idesc), "r"(accumulate)
+            : "memory");
+}
+
 // 128 lanes x 128 bits, shared memory -> tensor memory (4 columns).
 template <int CG>
 __device__ __forceinline__ void tmem_cp_128x128b(uint32_t taddr, uint64_t s_desc) {
@@ -409,6 +430,29 @@ __device__ __forceinline__ void ldg256_stream(const void* p, uint32_t (&r)[8]) {
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
                    "=r"(r[7])
                  : "l"(p));
+}
+// same 32-byte load with the default cache policy (the data is read again shortly)
+__device__ __forceinline__ void ldg256_keep(const void* p, uint32_t (&r)[8]) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+                   "=r"(r[7])
+                 : "l"(p));
+}
+__device__ __forceinline__ void stg128(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.global.v4.b32 [%4], {%0,%1,%2,%3};" ::"r"(a), "r"(b), "r"(c), "r"(d), "l"(p) : "memory");
+}
+// per-half unsigned maximum of two packed 16-bit pairs
+__device__ __forceinline__ uint32_t vmax_u16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// two fp32 -> two E4M3 codes (round to nearest even, finite overflow saturates to +-448):
+// `lo` in bits 0..7, `hi` in bits 8..15
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
+    uint16_t d;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    return (uint32_t)d;
 }
 __device__ __forceinline__ void stg256(void* p, const uint32_t (&r)[8]) {
     asm volatile("st.global.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};" ::"r"(r[0]), "r"(r[1]), "r"(r[2]),

@@ -47,6 +47,7 @@ struct GemmParams {
     const float* row_scale;    // [M] or nullptr
     const float* scale_partial;  // or: per-K-split row sums of a deferred prune launch (see
     int scale_ks;                //     row_scale_from_partials), scale_ks splits per 16-row block
+    const float* col_scale;      // [N] per-output-channel factor (FP8 weight scales) or nullptr
     const uint16_t* bias;      // [N] bf16 or nullptr
     const uint16_t* residual;  // [M x N] bf16 (ld = ldr) or nullptr
     int64_t ldr;
@@ -161,16 +162,24 @@ struct L0Schedule {
     }
 };
 
-template <int BN_, int CG_, int STAGES_, int CBUFS_>
+// FP8_ = true: E4M3 operands (one byte per element).  The byte geometry of a stage is the same
+// (a 128-byte swizzled row of compressed A is then 256 logical K instead of 128, a 128-byte row of
+// W 128 K instead of 64), the metadata of a stage doubles (two 128 x 128 blocks), and the four MMAs
+// of a stage are kind::f8f6f4 with K = 64 each.
+template <int BN_, int CG_, int STAGES_, int CBUFS_, bool FP8_ = false>
 struct GemmCfg {
     static constexpr int BN = BN_, CG = CG_, STAGES = STAGES_, CBUFS = CBUFS_;
+    static constexpr bool FP8 = FP8_;
     static constexpr int BM = 128;  // rows per CTA
-    static constexpr int BK = 128;  // logical K per stage
+    static constexpr int BK = FP8 ? 256 : 128;  // logical K per stage
+    static constexpr int A_BOX_X = FP8 ? 128 : 64;  // stored A elements per 128-byte row
+    static constexpr int B_BOX_X = FP8 ? 128 : 64;  // W elements per 128-byte row
     static constexpr int BN_CTA = BN / CG;
-    static constexpr int A_BYTES = BM * (BK / 2) * 2;     // 16 KB
-    static constexpr int B_HALF_BYTES = BN_CTA * 64 * 2;  // one 64-element K slice of the W tile
+    static constexpr int A_BYTES = BM * 128;              // 128 swizzled rows of 128 bytes: 16 KB
+    static constexpr int B_HALF_BYTES = BN_CTA * 128;     // one 128-byte K slice of the W tile
     static constexpr int B_BYTES = 2 * B_HALF_BYTES;
-    static constexpr int E_BYTES = 2048;
+    static constexpr int E_BYTES = FP8 ? 4096 : 2048;
+    static constexpr int E_COLS = E_BYTES / 512;  // tensor-memory columns of a stage's metadata
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
     // epilogue chunk: 64 columns (128-byte swizzled staging rows) when BN allows, else 48 columns
     // (96-byte unswizzled rows) -- BN = 240 is the widest tile that leaves room for two
@@ -178,7 +187,7 @@ struct GemmCfg {
     static constexpr int CH = (BN % 64 == 0) ? 64 : 48;
     static constexpr int C_BOX_BYTES = 32 * CH * 2;  // one warp's 32 x CH bf16 store box
     static constexpr int C_BYTES = 4 * CBUFS * C_BOX_BYTES;
-    static constexpr int ACC_STAGES = (2 * BN + 4 * STAGES <= 512) ? 2 : 1;
+    static constexpr int ACC_STAGES = (2 * BN + E_COLS * STAGES <= 512) ? 2 : 1;
     static constexpr int E_COL0 = ACC_STAGES * BN;  // metadata columns start after accumulators
     static constexpr int TMEM_COLS = 512;
     static constexpr int NUM_BARS = 2 * STAGES + 2 * ACC_STAGES;
@@ -188,14 +197,14 @@ struct GemmCfg {
     static_assert(BN % CH == 0, "epilogue works on whole chunks");
     static_assert(C_BOX_BYTES % 1024 == 0, "staging boxes stay 1024-byte aligned");
     static_assert(B_HALF_BYTES % 1024 == 0, "swizzle atoms need 1024-byte aligned tiles");
-    static_assert(E_COL0 % 4 == 0 && E_COL0 + 4 * STAGES <= TMEM_COLS, "tensor memory budget");
+    static_assert(E_COL0 % 4 == 0 && E_COL0 + E_COLS * STAGES <= TMEM_COLS, "tensor memory budget");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
     // phase 0 stage (rank 64): L_B boxes at the start of the W slot, second X box behind them
     static constexpr int L0_R = 64;
     static constexpr int L0_LB_BYTES = (L0_R / CG) * 64 * 2;
     static constexpr int L0_X2_OFF = (2 * L0_LB_BYTES + 1023) / 1024 * 1024;
     static constexpr int L0_STAGE_BYTES = 2 * A_BYTES + 2 * L0_LB_BYTES;
-    static constexpr bool L0_OK = L0_X2_OFF + A_BYTES <= B_BYTES;
+    static constexpr bool L0_OK = !FP8 && L0_X2_OFF + A_BYTES <= B_BYTES;
 };
 
 // Instruction descriptor of tcgen05.mma.sp kind::f16: bf16 x bf16 -> fp32, both operands
@@ -207,6 +216,10 @@ __host__ __device__ constexpr uint32_t make_idesc_sp_bf16(int m, int n) {
            | (1u << 10)                     // B format: bf16
            | ((uint32_t)(n >> 3) << 17)     // N / 8
            | ((uint32_t)(m >> 4) << 24);    // M / 16
+}
+// The same for kind::f8f6f4 with E4M3 operands (format code 0 in both operand fields).
+__host__ __device__ constexpr uint32_t make_idesc_sp_e4m3(int m, int n) {
+    return (1u << 2) | (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // LORA = false is the plain layer: the low-rank stages and phase 0 are compiled out, so the hot
@@ -292,6 +305,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             bool ok = true;
             bool l0_all_done = false;
             const uint32_t full0 = (CG == 2) ? mapa(bar_full, 0) : bar_full;  // leader's barriers
+            constexpr int E_ROWS = Cfg::E_BYTES / 1024;  // 1024-byte rows of the metadata tensor map per stage
             if constexpr (L0) {
                 // phase 0: dense X boxes and L_B boxes of this cluster's (row block, K split) items
                 for (int li = 0; li < l0_n && ok; ++li) {
@@ -345,19 +359,19 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     if constexpr (CG == 1) {
                         const uint32_t bar = bar_full + 8 * stage;
                         mbar_arrive_expect_tx(bar, Cfg::STAGE_BYTES);
-                        tma_load_2d(a_dst, &tmap_a, kb * 64, m0, bar);
-                        tma_load_2d(e_dst, &tmap_e, 0, 2 * (eblk + kb), bar);
-                        tma_load_2d(b_dst, &tmap_b, kb * 128, n0, bar);
-                        tma_load_2d(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * 128 + 64, n0, bar);
+                        tma_load_2d(a_dst, &tmap_a, kb * Cfg::A_BOX_X, m0, bar);
+                        tma_load_2d(e_dst, &tmap_e, 0, E_ROWS * (eblk + kb), bar);
+                        tma_load_2d(b_dst, &tmap_b, kb * Cfg::BK, n0, bar);
+                        tma_load_2d(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + Cfg::B_BOX_X, n0, bar);
                     } else {
                         const uint32_t bar = full0 + 8 * stage;
                         // the leader announces the bytes of both CTAs; the peer's bytes may land
                         // first (the count goes negative for a moment, which is allowed)
                         if (leader) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * Cfg::STAGE_BYTES);
-                        tma_load_2d_pair(a_dst, &tmap_a, kb * 64, m0, bar);
-                        tma_load_2d_pair(e_dst, &tmap_e, 0, 2 * (eblk + kb), bar);
-                        tma_load_2d_pair(b_dst, &tmap_b, kb * 128, n0, bar);
-                        tma_load_2d_pair(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * 128 + 64, n0, bar);
+                        tma_load_2d_pair(a_dst, &tmap_a, kb * Cfg::A_BOX_X, m0, bar);
+                        tma_load_2d_pair(e_dst, &tmap_e, 0, E_ROWS * (eblk + kb), bar);
+                        tma_load_2d_pair(b_dst, &tmap_b, kb * Cfg::BK, n0, bar);
+                        tma_load_2d_pair(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + Cfg::B_BOX_X, n0, bar);
                     }
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -471,16 +485,27 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t e_tmem = tmem_base + Cfg::E_COL0 + 4 * stage;
+                    const uint32_t e_tmem = tmem_base + Cfg::E_COL0 + Cfg::E_COLS * stage;
                     const uint32_t a_lo = a_lo0 + stage * (Cfg::A_BYTES >> 4);
                     const uint32_t b_lo = b_lo0 + stage * (Cfg::B_BYTES >> 4);
                     tmem_cp_128x128b<CG>(e_tmem, e_d0 + (uint64_t)(stage * (Cfg::E_BYTES >> 4)));
-                    // four K steps of 32 logical elements: A advances 32 bytes, W 64 bytes (steps 2, 3
-                    // in the second 64-element slice); metadata column pair + sparse_id2 = step parity
-                    mma_sp_bf16_lh<CG>(d_tmem, a_lo, b_lo, desc_hi, e_tmem, idesc0, accumulate);
-                    mma_sp_bf16_lh<CG>(d_tmem, a_lo + 2, b_lo + 4, desc_hi, e_tmem, idesc1, 1u);
-                    mma_sp_bf16_lh<CG>(d_tmem, a_lo + 4, b_lo + BH, desc_hi, e_tmem + 2, idesc0, 1u);
-                    mma_sp_bf16_lh<CG>(d_tmem, a_lo + 6, b_lo + BH + 4, desc_hi, e_tmem + 2, idesc1, 1u);
+                    if constexpr (Cfg::FP8) {
+                        // second 128 x 128 metadata block of the stage, then four K steps of 64 logical
+                        // elements: A advances 32 bytes, W 64 bytes, metadata two columns
+                        tmem_cp_128x128b<CG>(e_tmem + 4, e_d0 + (uint64_t)(stage * (Cfg::E_BYTES >> 4) + (2048 >> 4)));
+                        constexpr uint32_t idesc8 = make_idesc_sp_e4m3(Cfg::BM * CG, BN);
+                        mma_sp_f8_lh<CG>(d_tmem, a_lo, b_lo, desc_hi, e_tmem, idesc8, accumulate);
+                        mma_sp_f8_lh<CG>(d_tmem, a_lo + 2, b_lo + 4, desc_hi, e_tmem + 2, idesc8, 1u);
+                        mma_sp_f8_lh<CG>(d_tmem, a_lo + 4, b_lo + BH, desc_hi, e_tmem + 4, idesc8, 1u);
+                        mma_sp_f8_lh<CG>(d_tmem, a_lo + 6, b_lo + BH + 4, desc_hi, e_tmem + 6, idesc8, 1u);
+                    } else {
+                        // four K steps of 32 logical elements: A advances 32 bytes, W 64 bytes (steps 2, 3
+                        // in the second 64-element slice); metadata column pair + sparse_id2 = step parity
+                        mma_sp_bf16_lh<CG>(d_tmem, a_lo, b_lo, desc_hi, e_tmem, idesc0, accumulate);
+                        mma_sp_bf16_lh<CG>(d_tmem, a_lo + 2, b_lo + 4, desc_hi, e_tmem, idesc1, 1u);
+                        mma_sp_bf16_lh<CG>(d_tmem, a_lo + 4, b_lo + BH, desc_hi, e_tmem + 2, idesc0, 1u);
+                        mma_sp_bf16_lh<CG>(d_tmem, a_lo + 6, b_lo + BH + 4, desc_hi, e_tmem + 2, idesc1, 1u);
+                    }
                     accumulate = 1u;
                     if constexpr (CG == 1) tc_commit(bar_empty + 8 * stage);
                     else tc_commit_pair(bar_empty + 8 * stage, 0x3);
@@ -733,11 +758,20 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                             r[6] = bf16_lo_f(rv.w); r[7] = bf16_hi_f(rv.w);
                         }
                     }
+                    float cs[8] = {s, s, s, s, s, s, s, s};  // row scale (x per-channel weight scale)
+                    if constexpr (Cfg::FP8) {
+                        if (p.col_scale != nullptr && n < p.N) {
+                            const float4 c0 = __ldg(reinterpret_cast<const float4*>(p.col_scale + n));
+                            const float4 c1 = __ldg(reinterpret_cast<const float4*>(p.col_scale + n) + 1);
+                            cs[0] = s * c0.x; cs[1] = s * c0.y; cs[2] = s * c0.z; cs[3] = s * c0.w;
+                            cs[4] = s * c1.x; cs[5] = s * c1.y; cs[6] = s * c1.z; cs[7] = s * c1.w;
+                        }
+                    }
                     uint32_t o[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const float y0 = fmaf(s, __uint_as_float(v[j * 8 + 2 * e]), b[2 * e]) + r[2 * e];
-                        const float y1 = fmaf(s, __uint_as_float(v[j * 8 + 2 * e + 1]), b[2 * e + 1]) + r[2 * e + 1];
+                        const float y0 = fmaf(cs[2 * e], __uint_as_float(v[j * 8 + 2 * e]), b[2 * e]) + r[2 * e];
+                        const float y1 = fmaf(cs[2 * e + 1], __uint_as_float(v[j * 8 + 2 * e + 1]), b[2 * e + 1]) + r[2 * e + 1];
                         o[e] = pack_bf16x2(y0, y1);
                     }
                     if constexpr (CH == 64)  // 128-byte rows, 16-byte chunk index XOR (row % 8): the 128-byte swizzle
