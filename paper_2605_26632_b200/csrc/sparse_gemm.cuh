@@ -192,7 +192,14 @@ struct GemmCfg {
     static constexpr int TMEM_COLS = 512;
     static constexpr int NUM_BARS = 2 * STAGES + 2 * ACC_STAGES;
     static constexpr int SMEM_BYTES = 1024 /*align slack*/ + STAGES * STAGE_BYTES + C_BYTES + 256;
-    static constexpr int THREADS = 192;
+    // Epilogue warps: four (one per tensor-memory lane quarter), or eight for FP8 -- two per quarter
+    // that take alternate column chunks, each with one staging box.  A tile's epilogue takes ~6 us
+    // with four warps, which an FP8 main loop at K = 3072 (6.5 us) no longer hides.
+    static constexpr int EPI_WARPS = FP8 ? 8 : 4;
+    static constexpr int EPI_SPLIT = EPI_WARPS / 4;          // warps per lane quarter
+    static constexpr int CBUFS_W = 4 * CBUFS / EPI_WARPS;    // staging boxes per epilogue warp
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;
+    static_assert(CBUFS_W >= 1, "every epilogue warp needs a staging box");
     static_assert(BN % 16 == 0 && (BN / CG) % 8 == 0 && BN <= 256, "tile N");
     static_assert(BN % CH == 0, "epilogue works on whole chunks");
     static_assert(C_BOX_BYTES % 1024 == 0, "staging boxes stay 1024-byte aligned");
@@ -269,7 +276,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         }
         for (int a = 0; a < Cfg::ACC_STAGES; ++a) {
             mbar_init(bar_tfull + 8 * a, 1);         // one tcgen05.commit
-            mbar_init(bar_tempty + 8 * a, 4 * CG);   // one arrive per epilogue warp of the pair
+            mbar_init(bar_tempty + 8 * a, Cfg::EPI_WARPS * CG);  // one arrive per epilogue warp of the pair
         }
         fence_mbar_init();
         prefetch_tmap(&tmap_a);
@@ -540,7 +547,8 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     } else {
         // ------------------------------------------------------------------ epilogue ----------
         const int q = warp & 3;  // tensor-memory lane quarter this warp may read
-        const uint32_t cbuf0 = sC + (warp - 2) * Cfg::CBUFS * Cfg::C_BOX_BYTES;
+        const uint32_t cbuf0 = sC + (warp - 2) * Cfg::CBUFS_W * Cfg::C_BOX_BYTES;
+        const int c_first = (warp - 2) >> 2;  // with two warps per quarter: even or odd chunks
         const uint32_t tempty0 = (CG == 2) ? mapa(bar_tempty, 0) : bar_tempty;
         int it = 0, cb = 0;
         bool alive = true;
@@ -663,6 +671,24 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 if (p.scale_partial != nullptr) s = row_scale_from_partials(p.scale_partial, row, p.scale_ks);
                 else if (p.row_scale != nullptr) s = __ldg(p.row_scale + row);
             }
+            // the tile's per-column terms (bias, FP8 weight scale), one column per lane and round,
+            // fetched while the main loop runs and handed round by shuffles in the chunk loop: no
+            // dependent global load is left between the accumulator and the store
+            constexpr int CH = Cfg::CH;
+            float bl_all[BN / CH][2], cl_all[BN / CH][2];
+#pragma unroll
+            for (int c = 0; c < BN / CH; ++c)
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int idx = u * 32 + lane, n = tn * BN + c * CH + idx;
+                    bl_all[c][u] = 0.f;
+                    cl_all[c][u] = 1.f;
+                    if (idx < CH && n < p.N) {
+                        if (p.bias != nullptr) bl_all[c][u] = __uint_as_float((uint32_t)__ldg(p.bias + n) << 16);
+                        if constexpr (Cfg::FP8)
+                            if (p.col_scale != nullptr) cl_all[c][u] = __ldg(p.col_scale + n);
+                    }
+                }
             if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, cta_abort, p.dev_error)) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
@@ -683,10 +709,22 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
                 if (!alive) break;
             }
-            constexpr int CH = Cfg::CH;
+            constexpr int NCH = BN / CH;
+            // this warp's last chunk: after reading it the accumulator goes back to the issuer
+            const int c_last = NCH - 1 - ((NCH - 1 - c_first) % Cfg::EPI_SPLIT);
 #pragma unroll 1
-            for (int c = 0; c < BN / CH; ++c) {
+            for (int c = c_first; c < NCH; c += Cfg::EPI_SPLIT) {
                 const int n0 = tn * BN + c * CH;
+                // this chunk's two rounds, picked with selects so that the arrays stay in registers
+                // (an index that depends on the loop counter would put them into local memory and
+                // force every load above to complete before the wait)
+                float bl[2] = {bl_all[0][0], bl_all[0][1]}, cl[2] = {cl_all[0][0], cl_all[0][1]};
+#pragma unroll
+                for (int cc = 1; cc < BN / CH; ++cc)
+                    if (c == cc) {
+                        bl[0] = bl_all[cc][0]; bl[1] = bl_all[cc][1];
+                        cl[0] = cl_all[cc][0]; cl[1] = cl_all[cc][1];
+                    }
                 uint32_t v[CH];
                 tmem_ld_32x32b_x32(t_row + c * CH, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
                 if constexpr (CH == 64)
@@ -694,7 +732,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 else
                     tmem_ld_32x32b_x16(t_row + c * CH + 32, *reinterpret_cast<uint32_t(*)[16]>(&v[32]));
                 tmem_ld_wait();
-                if (c == BN / CH - 1) {
+                if (c == c_last) {
                     // accumulator fully read: hand it back to the MMA issuer
                     tc_fence_before();
                     __syncwarp();
@@ -734,22 +772,20 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 }
                 if (n0 >= p.N) continue;
                 // staging buffer must have been read by its previous TMA store
-                if (lane == 0) tma_store_wait_read<Cfg::CBUFS - 1>();
+                if (lane == 0) tma_store_wait_read<Cfg::CBUFS_W - 1>();
                 __syncwarp();
                 const uint32_t cbuf = cbuf0 + cb * Cfg::C_BOX_BYTES;
 #pragma unroll
                 for (int j = 0; j < CH / 8; ++j) {  // 8 columns (16 bytes of output) at a time
                     const int n = n0 + j * 8;
-                    float b[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    float b[8];
                     float r[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int col = j * 8 + e;
+                        b[e] = __shfl_sync(0xffffffffu, bl[col >> 5], col & 31);
+                    }
                     if (n < p.N) {
-                        if (p.bias != nullptr) {
-                            const uint4 bv = __ldg(reinterpret_cast<const uint4*>(p.bias + n));
-                            b[0] = bf16_lo_f(bv.x); b[1] = bf16_hi_f(bv.x);
-                            b[2] = bf16_lo_f(bv.y); b[3] = bf16_hi_f(bv.y);
-                            b[4] = bf16_lo_f(bv.z); b[5] = bf16_hi_f(bv.z);
-                            b[6] = bf16_lo_f(bv.w); b[7] = bf16_hi_f(bv.w);
-                        }
                         if (p.residual != nullptr && row_ok) {
                             const uint4 rv = __ldg(reinterpret_cast<const uint4*>(p.residual + row * p.ldr + n));
                             r[0] = bf16_lo_f(rv.x); r[1] = bf16_hi_f(rv.x);
@@ -760,11 +796,10 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     }
                     float cs[8] = {s, s, s, s, s, s, s, s};  // row scale (x per-channel weight scale)
                     if constexpr (Cfg::FP8) {
-                        if (p.col_scale != nullptr && n < p.N) {
-                            const float4 c0 = __ldg(reinterpret_cast<const float4*>(p.col_scale + n));
-                            const float4 c1 = __ldg(reinterpret_cast<const float4*>(p.col_scale + n) + 1);
-                            cs[0] = s * c0.x; cs[1] = s * c0.y; cs[2] = s * c0.z; cs[3] = s * c0.w;
-                            cs[4] = s * c1.x; cs[5] = s * c1.y; cs[6] = s * c1.z; cs[7] = s * c1.w;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const int col = j * 8 + e;
+                            cs[e] = s * __shfl_sync(0xffffffffu, cl[col >> 5], col & 31);
                         }
                     }
                     uint32_t o[4];
@@ -785,7 +820,7 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     tma_store_2d(&tmap_y, n0, m0, cbuf);
                     tma_store_commit();
                 }
-                cb = (cb + 1 == Cfg::CBUFS) ? 0 : cb + 1;
+                cb = (cb + 1 == Cfg::CBUFS_W) ? 0 : cb + 1;
             }
             if (w.kind == 1) {
                 // publish: all lanes' stores (ordered before lane 0 by the warp barrier), then the

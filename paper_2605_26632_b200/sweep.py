@@ -66,6 +66,9 @@ def main():
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--no-fused", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph replay")
+    ap.add_argument("--fp8", action="store_true",
+                    help="time the FP8 (E4M3) composition instead: quantising prune, FP8 sparse GEMM, the FP8 layer, "
+                         "next to the bf16 sparse layer, the dense bf16 linear and torch's dense FP8 GEMM")
     ap.add_argument("--lora", type=int, default=0, metavar="R",
                     help="time the low-rank branch of rank R instead: down projection alone, layer with it, "
                          "and the dense linear followed by the two dense low-rank GEMMs of torch")
@@ -79,6 +82,8 @@ def main():
     shapes += [(inputs.OTHER_FAMILY_M, K, N) for (K, N) in inputs.OTHER_FAMILY_KN]
     if not args.quick:
         shapes += [(M, K, M) for M in (2048, 4096, 8192) for K in (3072, 12288)]  # the paper's kernel grid
+    if args.fp8:
+        return fp8_sweep(lx, shapes, args.iters)
     if args.lora:
         return lora_sweep(lx, shapes, args.lora, args.iters)
     print("| M | K | N | prune us | prune GB/s | GEMM us | GEMM TF | layer us | layer TF | fused us | fused TF | "
@@ -113,6 +118,46 @@ def main():
               f"{td/tg:.2f} | {td/tl:.2f} |", flush=True)
         assert lx.last_error() == 0
         del Xs, Ws, vs, ms, ss, Ys
+        torch.cuda.empty_cache()
+
+
+def fp8_sweep(lx, shapes, iters):
+    print("| M | K | N | prune fp8 us | GEMM fp8 us | GEMM fp8 TF | layer fp8 us | layer bf16 us | dense bf16 us | "
+          "dense fp8 (torch) us | fp8 layer / bf16 layer | fp8 layer / dense bf16 | fp8 layer / dense fp8 |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for (M, K, N) in shapes:
+        if K % 256:
+            continue
+        per_set = M * K * 2 + M * K + M * K // 8 + N * K * 2 + M * N * 2
+        nsets = max(2, math.ceil(400e6 / per_set))
+        g = torch.Generator(device="cuda").manual_seed(M + K + N)
+        Xs = [torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16) for _ in range(nsets)]
+        Ws = [(torch.randn(N, K, device="cuda", generator=g) * K ** -0.5).to(torch.bfloat16) for _ in range(nsets)]
+        b = torch.zeros(N, device="cuda", dtype=torch.bfloat16)
+        Ys = [torch.empty(M, N, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+        lx.reserve(M, N, K)
+        Wqs = [lx.quantize_weights_fp8(W, True) for W in Ws]
+        cs = [lx.prune_compress_fp8(X, 1) for X in Xs]
+        tp = timeloop(lambda j: lx.prune_compress_fp8(Xs[j], 1, *cs[j]), nsets, iters)
+        tg = timeloop(lambda j: lx.sparse_linear_fp8(cs[j][0], cs[j][1], Wqs[j][0], Wqs[j][1], b, cs[j][2], None, Ys[j]),
+                      nsets, iters)
+        tl = timeloop(lambda j: lx.act_sparse_linear_fp8(Xs[j], Wqs[j][0], Wqs[j][1], b, 1, None, Ys[j]), nsets, iters)
+        tb = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_SEPARATE), nsets, iters)
+        td = timeloop(lambda j: torch.nn.functional.linear(Xs[j], Ws[j], b), nsets, iters)
+        # torch's dense FP8 GEMM (cuBLASLt) on pre-quantised operands, per-tensor scales
+        Xq = [X.to(torch.float8_e4m3fn) for X in Xs]
+        Wt = [W.to(torch.float8_e4m3fn) for W in Ws]
+        one = torch.ones((), device="cuda", dtype=torch.float32)
+        try:
+            t8 = timeloop(lambda j: torch._scaled_mm(Xq[j], Wt[j].t(), scale_a=one, scale_b=one, bias=b,
+                                                     out_dtype=torch.bfloat16), nsets, iters)
+        except Exception:
+            t8 = float("nan")
+        fl = 2.0 * M * N * K
+        print(f"| {M} | {K} | {N} | {tp*1e3:.1f} | {tg*1e3:.1f} | {fl/tg/1e9:.0f} | {tl*1e3:.1f} | {tb*1e3:.1f} | "
+              f"{td*1e3:.1f} | {t8*1e3:.1f} | {tb/tl:.2f} | {td/tl:.2f} | {t8/tl:.2f} |", flush=True)
+        assert lx.last_error() == 0
+        del Xs, Ws, Ys, Wqs, cs, Xq, Wt
         torch.cuda.empty_cache()
 
 
