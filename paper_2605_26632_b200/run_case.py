@@ -1,6 +1,6 @@
 """Runs a few launches of one kernel of the path on a named synthetic workload.
 
-    python -m paper_2605_26632_b200.run_case --kernel prune|gemm|layer|fused|lora_down|lora_layer --workload mlp_down [--iters 3]
+    python -m paper_2605_26632_b200.run_case --kernel prune|gemm|layer|fused|lora_down|lora_layer|fp8_prune|fp8_gemm|fp8_layer --workload mlp_down [--iters 3]
 
 Meant as the small, self-terminating command to put under a profiler (one kernel, a few launches,
 well under a GB on the device), and as a minimal usage example of the binding.
@@ -16,7 +16,8 @@ from . import binding, inputs
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="layer", choices=["prune", "gemm", "layer", "fused", "lora_down", "lora_layer"])
+    ap.add_argument("--kernel", default="layer", choices=["prune", "gemm", "layer", "fused", "lora_down", "lora_layer", "fp8_prune", "fp8_gemm",
+                             "fp8_layer"])
     ap.add_argument("--rank", type=int, default=64, help="rank R of the low-rank branch")
     ap.add_argument("--workload", default="mlp_down")
     ap.add_argument("--M", type=int, default=0, help="override the number of token rows")
@@ -40,7 +41,16 @@ def main():
     T = torch.empty(M, R, device="cuda", dtype=torch.bfloat16)
     if args.kernel.startswith("lora"):
         lx.reserve_lora(M, wl.K, R)
+    if args.kernel.startswith("fp8"):
+        Wq, ws = lx.quantize_weights_fp8(W, per_channel=True)
+        vq, meta8, rs = lx.prune_compress_fp8(X, args.comp)
     for _ in range(args.iters):
+        if args.kernel == "fp8_prune":
+            lx.prune_compress_fp8(X, args.comp, vq, meta8, rs)
+        if args.kernel == "fp8_gemm":
+            lx.sparse_linear_fp8(vq, meta8, Wq, ws, b, rs, None, Y)
+        if args.kernel == "fp8_layer":
+            lx.act_sparse_linear_fp8(X, Wq, ws, b, args.comp, None, Y)
         if args.kernel in ("prune", "layer"):
             lx.prune_compress(X, args.comp, values, meta, scale)
         if args.kernel in ("gemm", "layer"):
