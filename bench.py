@@ -317,7 +317,7 @@ def main():
     gemm_ms = [evs[i][1].elapsed_time(evs[i][2]) for i in probed]
 
     # prune/compress (row scale finalized in the same launch) alone, back to back over the rotating sets: the
-    # per-launch time that the HBM roofline of that kernel is judged on
+    # per-launch time that the HBM roofline of that kernel is computed from
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for i in range(3):
         lx.prune_compress(Xs[i % NSETS], comp_mode, vals[i % NSETS], metas[i % NSETS], scales[i % NSETS] if comp_mode else None)
