@@ -270,13 +270,15 @@ def quantize_weights_fp8(W, per_channel: bool):
     return Wq, ws
 
 
-def compress_fp8(X):
-    """-> (values_q uint8 [M, K/2], meta_canon uint16 [M, K/16], act_scale float32 [M])"""
+def compress_fp8(X, row_amax=None):
+    """-> (values_q uint8 [M, K/2], meta_canon uint16 [M, K/16], act_scale float32 [M]);
+    row_amax (float32 [M]) replaces the row maxima taken from the data."""
     X, M, K = _check_x(X)
+    row_amax = None if row_amax is None else np.ascontiguousarray(row_amax, dtype=np.float32)
     vq = np.empty((M, K // 2), dtype=np.uint8)
     meta = np.empty((M, K // 16), dtype=np.uint16)
     sc = np.empty(M, dtype=np.float32)
-    _load().oracle_compress_fp8(_p(X), _i64(M), _i64(K), _i64(K), _p(vq), _p(meta), _p(sc))
+    _load().oracle_compress_fp8(_p(X), _i64(M), _i64(K), _i64(K), _p(row_amax), _p(vq), _p(meta), _p(sc))
     return vq, meta, sc
 
 
@@ -287,7 +289,7 @@ def meta_canon_to_hw_fp8(meta_canon, M: int, K: int) -> np.ndarray:
     return out
 
 
-def act_sparse_linear_fp8(X, Wq, wscale, bias=None, comp_mode=COMP_NONE, Yr=None, rows=None):
+def act_sparse_linear_fp8(X, Wq, wscale, bias=None, comp_mode=COMP_NONE, Yr=None, rows=None, row_amax=None):
     """Whole FP8 path.  -> dict(values_q, meta_canon, row_scale (= s * act_scale), Y[fp32, rows x N])."""
     X, M, K = _check_x(X)
     Wq = np.ascontiguousarray(Wq, dtype=np.uint8)
@@ -302,7 +304,8 @@ def act_sparse_linear_fp8(X, Wq, wscale, bias=None, comp_mode=COMP_NONE, Yr=None
     rs = np.empty(M, dtype=np.float32)
     acc = np.empty((nr, N), dtype=np.float32)
     Y = np.empty((nr, N), dtype=np.float32)
-    _load().oracle_act_sparse_linear_fp8(_p(X), _i64(M), _i64(K), _i64(K), _p(Wq), _p(wscale), _i64(N), _p(bias),
+    row_amax = None if row_amax is None else np.ascontiguousarray(row_amax, dtype=np.float32)
+    _load().oracle_act_sparse_linear_fp8(_p(X), _i64(M), _i64(K), _i64(K), _p(row_amax), _p(Wq), _p(wscale), _i64(N), _p(bias),
                                          ctypes.c_int(comp_mode), _p(Yr), _i64(N), _p(r), _i64(nr), _p(vq),
                                          _p(meta), _p(rs), _p(acc), _p(Y))
     return {"values_q": vq, "meta_canon": meta, "row_scale": rs, "Y": Y}

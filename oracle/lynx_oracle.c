@@ -503,16 +503,19 @@ ORACLE_API void oracle_quantize_weights_fp8(const uint16_t* W, int64_t N, int64_
 }
 
 /* Activations: Top-2-of-4 on the bf16 values, then per-row symmetric FP8 codes of the kept ones.
- * values_q [M x K/2] codes, meta_canon as oracle_compress, act_scale [M]. */
-ORACLE_API void oracle_compress_fp8(const uint16_t* X, int64_t M, int64_t K, int64_t ldx, uint8_t* values_q,
-                                    uint16_t* meta_canon, float* act_scale) {
+ * values_q [M x K/2] codes, meta_canon as oracle_compress, act_scale [M].
+ * row_amax: NULL = the row maximum is taken from the data; else row_amax[m] is used in its place
+ * (a scale calibrated beforehand, or a maximum the producer of X already knows); values beyond
+ * it saturate. */
+ORACLE_API void oracle_compress_fp8(const uint16_t* X, int64_t M, int64_t K, int64_t ldx, const float* row_amax,
+                                    uint8_t* values_q, uint16_t* meta_canon, float* act_scale) {
     const int64_t G = K / 4;
     memset(meta_canon, 0, (size_t)(M * (K / 16)) * sizeof(uint16_t));
     for (int64_t m = 0; m < M; ++m) {
         unsigned top = 0;
         for (int64_t k = 0; k < K; ++k)
             if (mag15(X[m * ldx + k]) > top) top = mag15(X[m * ldx + k]);
-        const float amax = bf16_to_f32((uint16_t)top);
+        const float amax = row_amax ? row_amax[m] : bf16_to_f32((uint16_t)top);
         const float inv = amax > 0.0f ? 448.0f / amax : 0.0f;  /* 0 for amax = 0 and for NaN */
         act_scale[m] = amax / 448.0f;
         for (int64_t g = 0; g < G; ++g) {
@@ -553,14 +556,14 @@ ORACLE_API void oracle_gemm_fp8_f32(const uint8_t* values_q, const uint16_t* met
 /* Whole FP8 path for a set of rows.  comp_mode: 0 none, 1 per-row norm compensation.
  * row_scale_out[m] = s_m * act_scale_m (what the epilogue multiplies row m by). */
 ORACLE_API void oracle_act_sparse_linear_fp8(const uint16_t* X, int64_t M, int64_t K, int64_t ldx,
-                                             const uint8_t* Wq, const float* wscale, int64_t N,
+                                             const float* row_amax, const uint8_t* Wq, const float* wscale, int64_t N,
                                              const uint16_t* bias, int comp_mode, const uint16_t* Yr, int64_t ldr,
                                              const int64_t* rows, int64_t n_rows, uint8_t* values_q,
                                              uint16_t* meta_canon, float* row_scale_out, float* acc_scratch,
                                              float* Y) {
     float* act = (float*)malloc((size_t)M * sizeof(float));
     float* s = (float*)malloc((size_t)M * sizeof(float));
-    oracle_compress_fp8(X, M, K, ldx, values_q, meta_canon, act);
+    oracle_compress_fp8(X, M, K, ldx, row_amax, values_q, meta_canon, act);
     oracle_row_scale(X, M, K, ldx, comp_mode == 1 ? 1 : 0, s);
     for (int64_t m = 0; m < M; ++m) row_scale_out[m] = s[m] * act[m];
     oracle_gemm_fp8_f32(values_q, meta_canon, M, K, Wq, N, rows, n_rows, acc_scratch);

@@ -456,6 +456,24 @@ def test_fp8_activation_codes_closed_forms():
     assert (err <= np.maximum(np.abs(kept) * 2.0 ** -4, sc[:, None] * 2.0 ** -10) * 1.0001).all()
 
 
+def test_fp8_given_row_maximum():
+    """A supplied maximum equal to the true one changes nothing; a larger one scales the codes
+    down (same mask); a smaller one saturates at +-448."""
+    g = torch.Generator().manual_seed(36)
+    M, K = 8, 256
+    x = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    X = inputs.as_u16(x)
+    vq, meta, sc = oracle.compress_fp8(X)
+    amax = x.float().abs().max(dim=1).values.numpy()
+    vq1, meta1, sc1 = oracle.compress_fp8(X, row_amax=amax)
+    assert (vq1 == vq).all() and (meta1 == meta).all() and (sc1 == sc).all()
+    vq2, meta2, sc2 = oracle.compress_fp8(X, row_amax=2 * amax)
+    assert (meta2 == meta).all() and (sc2 == 2 * sc).all()
+    assert np.abs(oracle.e4m3_decode(vq2)).max() == 224.0
+    vq3, _, sc3 = oracle.compress_fp8(X, row_amax=0.25 * amax)
+    assert np.abs(oracle.e4m3_decode(vq3)).max() == 448.0 and (np.abs(oracle.e4m3_decode(vq3)) == 448.0).sum() > M
+
+
 def test_fp8_metadata_order_is_the_rows_bytes_block_by_block():
     """Independent restatement: per (128-row, 128-K) block, row r's 16 bytes are the row's 8
     canonical little-endian words of that K block; rows past M are 0x44."""
