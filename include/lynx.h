@@ -262,22 +262,27 @@ LYNX_API lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, i
  * lynx_meta_bytes(M, K) but its own order: blocks of 128 rows x 128 K-elements, 2048 bytes each,
  * block (rb, kb) at byte (rb * K/128 + kb) * 2048, inside a block row r's 16 bytes at r * 16 with
  * group g = (k % 128) / 4 in bits 4 * (g % 2) of byte g / 2; rows past M hold 0x4 nibbles.
- * lynx_prune_compress_fp8 reads X twice (row maxima first; the second pass normally hits the L2)
- * and needs no scratch.  The low-rank branch, LYNX_COMP_TENSOR / GROUP and the one-kernel mode are
+ * row_amax (optional, [M] fp32 on the device): when given, row_amax[m] takes the place of the
+ * row maximum found in the data -- a scale calibrated beforehand (the same number in every entry)
+ * or a maximum the producer of X already knows; values beyond it saturate at +-448.  Without it
+ * lynx_prune_compress_fp8 reads X twice (row maxima first; the second pass normally hits the L2),
+ * with it once.  Neither form needs scratch.  The low-rank branch, LYNX_COMP_TENSOR / GROUP and the one-kernel mode are
  * not available in FP8.
  */
 LYNX_API lynx_status lynx_quantize_weights_fp8(lynx_ctx* ctx, const void* W, int64_t N, int64_t K,
                                                int64_t ldw, int per_channel, void* Wq, float* wscale,
                                                void* stream);
 LYNX_API lynx_status lynx_prune_compress_fp8(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
-                                             int64_t ldx, void* values_q, void* meta,
-                                             float* row_scale, lynx_comp_mode mode, void* stream);
+                                             int64_t ldx, const float* row_amax, void* values_q,
+                                             void* meta, float* row_scale, lynx_comp_mode mode,
+                                             void* stream);
 LYNX_API lynx_status lynx_sparse_linear_fp8(lynx_ctx* ctx, const void* values_q, const void* meta,
                                             int64_t M, int64_t K, const void* Wq, int64_t N,
                                             int64_t ldwq, const float* wscale, const void* bias,
                                             const lynx_comp* comp, void* Y, int64_t ldy, void* stream);
 LYNX_API lynx_status lynx_act_sparse_linear_fp8(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
-                                                int64_t ldx, const void* Wq, int64_t N, int64_t ldwq,
+                                                int64_t ldx, const float* row_amax, const void* Wq,
+                                                int64_t N, int64_t ldwq,
                                                 const float* wscale, const void* bias,
                                                 lynx_comp_mode mode, const void* residual, int64_t ldr,
                                                 void* Y, int64_t ldy, void* stream);

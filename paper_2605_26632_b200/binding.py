@@ -82,11 +82,11 @@ def load_library() -> ctypes.CDLL:
     lib.lynx_act_sparse_linear_lora.argtypes = [vp, vp, i64, i64, i64, vp, i64, i64, vp, vp, i64, vp, i64, i64,
                                                 i32, vp, i64, vp, i64, vp]
     lib.lynx_quantize_weights_fp8.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp]
-    lib.lynx_prune_compress_fp8.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, i32, vp]
+    lib.lynx_prune_compress_fp8.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, vp, i32, vp]
     lib.lynx_sparse_linear_fp8.argtypes = [vp, vp, vp, i64, i64, vp, i64, i64, vp, vp, ctypes.POINTER(_Comp), vp,
                                            i64, vp]
-    lib.lynx_act_sparse_linear_fp8.argtypes = [vp, vp, i64, i64, i64, vp, i64, i64, vp, vp, i32, vp, i64, vp, i64,
-                                               vp]
+    lib.lynx_act_sparse_linear_fp8.argtypes = [vp, vp, i64, i64, i64, vp, vp, i64, i64, vp, vp, i32, vp, i64, vp,
+                                               i64, vp]
     lib.lynx_launch_count.argtypes = [vp]
     lib.lynx_launch_count.restype = i64
     _lib = lib
@@ -304,8 +304,10 @@ class Lynx:
                                                    _ptr(Wq), _ptr(ws), _stream()), "lynx_quantize_weights_fp8")
         return Wq, ws
 
-    def prune_compress_fp8(self, X: torch.Tensor, mode: int = COMP_NONE, values_q=None, meta=None, row_scale=None):
-        """-> (values_q uint8 [M, K/2], meta uint8, row_scale float32 [M] = s * amax / 448)"""
+    def prune_compress_fp8(self, X: torch.Tensor, mode: int = COMP_NONE, values_q=None, meta=None, row_scale=None,
+                           row_amax=None):
+        """-> (values_q uint8 [M, K/2], meta uint8, row_scale float32 [M] = s * amax / 448);
+        row_amax (float32 [M]) replaces the row maxima found in the data (X is then read once)."""
         _bf16_2d(X, "X")
         M, K = X.shape
         if values_q is None:
@@ -314,8 +316,9 @@ class Lynx:
             meta = torch.empty(meta_bytes(M, K), dtype=torch.uint8, device=X.device)
         if row_scale is None:
             row_scale = torch.empty(M, dtype=torch.float32, device=X.device)
-        _check(self._lib.lynx_prune_compress_fp8(self._h, _ptr(X), M, K, X.stride(0), _ptr(values_q), _ptr(meta),
-                                                 _ptr(row_scale), mode, _stream()), "lynx_prune_compress_fp8")
+        _check(self._lib.lynx_prune_compress_fp8(self._h, _ptr(X), M, K, X.stride(0), _ptr(row_amax), _ptr(values_q),
+                                                 _ptr(meta), _ptr(row_scale), mode, _stream()),
+               "lynx_prune_compress_fp8")
         return values_q, meta, row_scale
 
     def sparse_linear_fp8(self, values_q: torch.Tensor, meta: torch.Tensor, Wq: torch.Tensor, wscale=None,
@@ -333,13 +336,14 @@ class Lynx:
         return out
 
     def act_sparse_linear_fp8(self, X: torch.Tensor, Wq: torch.Tensor, wscale=None, bias=None,
-                              mode: int = COMP_NONE, residual=None, out=None) -> torch.Tensor:
+                              mode: int = COMP_NONE, residual=None, out=None, row_amax=None) -> torch.Tensor:
         _bf16_2d(X, "X")
         M, K = X.shape
         N = Wq.shape[0]
         if out is None:
             out = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
-        _check(self._lib.lynx_act_sparse_linear_fp8(self._h, _ptr(X), M, K, X.stride(0), _ptr(Wq), N, Wq.stride(0),
+        _check(self._lib.lynx_act_sparse_linear_fp8(self._h, _ptr(X), M, K, X.stride(0), _ptr(row_amax), _ptr(Wq), N,
+                                                    Wq.stride(0),
                                                     _ptr(wscale), _ptr(bias), mode, _ptr(residual),
                                                     0 if residual is None else residual.stride(0), _ptr(out),
                                                     out.stride(0), _stream()), "lynx_act_sparse_linear_fp8")

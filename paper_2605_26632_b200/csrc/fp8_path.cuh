@@ -75,10 +75,13 @@ __device__ __forceinline__ void quantize_kept16(const uint32_t* v /*[8]*/, float
 // Metadata block (rb, kb) of 128 rows x 128 K at byte (rb * K/128 + kb) * 2048; inside it row r's
 // 16 bytes at r * 16, group g = (k % 128) / 4 in bits 4 * (g % 2) of byte g / 2 (natural order).
 // mode: 0 -> row_scale = amax / 448; 1 -> row_scale = sqrt(sum x^2 / (sum kept^2 + 1e-8)) * amax / 448.
-template <bool SUMS>
+// GIVEN: the row maxima come from the caller (row_amax[m]: a calibrated scale, or a maximum the
+// producer of X already knows) and pass 1 is skipped: X is then read once.
+template <bool SUMS, bool GIVEN>
 __global__ void __launch_bounds__(FP8_PRUNE_WARPS * 32, 1)
 prune_compress_fp8_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int64_t ldx,
-                          uint8_t* __restrict__ values_q, uint8_t* __restrict__ meta, float* __restrict__ row_scale) {
+                          const float* __restrict__ row_amax, uint8_t* __restrict__ values_q,
+                          uint8_t* __restrict__ meta, float* __restrict__ row_scale) {
     __shared__ uint32_t lut[4 * 16];
     __shared__ uint32_t s_top[FP8_PRUNE_WARPS][16];
     __shared__ float2 s_sum[FP8_PRUNE_WARPS][16];
@@ -96,7 +99,7 @@ prune_compress_fp8_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, 
 
     // ---- pass 1: largest magnitude of each row (packed 16-bit maxima over the 15 magnitude bits)
     uint32_t mA = 0, mB = 0;
-    for (int t = warp; t < kb128; t += FP8_PRUNE_WARPS) {
+    for (int t = warp; !GIVEN && t < kb128; t += FP8_PRUNE_WARPS) {
         uint32_t a0[8], a1[8], b0[8], b1[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) a0[i] = a1[i] = b0[i] = b1[i] = 0u;
@@ -132,7 +135,11 @@ prune_compress_fp8_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, 
         topA = max(topA, s_top[w][r]);
         topB = max(topB, s_top[w][r + 8]);
     }
-    const float amaxA = __uint_as_float(topA << 16), amaxB = __uint_as_float(topB << 16);
+    float amaxA = __uint_as_float(topA << 16), amaxB = __uint_as_float(topB << 16);
+    if constexpr (GIVEN) {
+        amaxA = okA ? __ldg(row_amax + rowA) : 0.0f;
+        amaxB = okB ? __ldg(row_amax + rowB) : 0.0f;
+    }
     const float invA = amaxA > 0.0f ? __fdiv_rn(448.0f, amaxA) : 0.0f;
     const float invB = amaxB > 0.0f ? __fdiv_rn(448.0f, amaxB) : 0.0f;
 
@@ -177,7 +184,7 @@ prune_compress_fp8_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, 
         uint32_t top = 0;
 #pragma unroll
         for (int w = 0; w < FP8_PRUNE_WARPS; ++w) top = max(top, s_top[w][tid]);
-        float sc = __fdiv_rn(__uint_as_float(top << 16), 448.0f);
+        float sc = __fdiv_rn(GIVEN ? __ldg(row_amax + row0 + tid) : __uint_as_float(top << 16), 448.0f);
         if constexpr (SUMS) {
             float num = 0.f, den = 0.f;
 #pragma unroll

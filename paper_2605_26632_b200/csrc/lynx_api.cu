@@ -1025,8 +1025,9 @@ lynx_status lynx_quantize_weights_fp8(lynx_ctx* ctx, const void* W, int64_t N, i
     return cuda_ok(cudaGetLastError());
 }
 
-lynx_status lynx_prune_compress_fp8(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, void* values_q,
-                                    void* meta, float* row_scale, lynx_comp_mode mode, void* stream) {
+lynx_status lynx_prune_compress_fp8(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx,
+                                    const float* row_amax, void* values_q, void* meta, float* row_scale,
+                                    lynx_comp_mode mode, void* stream) {
     lynx_status s = check_fp8_shape(ctx, M, K);
     if (s != LYNX_OK) return s;
     if (!X || !values_q || !meta || !row_scale) return LYNX_ERR_INVALID_ARG;
@@ -1047,9 +1048,15 @@ lynx_status lynx_prune_compress_fp8(lynx_ctx* ctx, const void* X, int64_t M, int
     const uint16_t* Xp = static_cast<const uint16_t*>(X);
     uint8_t* vp = static_cast<uint8_t*>(values_q);
     uint8_t* mp = static_cast<uint8_t*>(meta);
-    cudaError_t e = (mode == LYNX_COMP_ROW)
-                        ? cudaLaunchKernelEx(&pc, prune_compress_fp8_kernel<true>, Xp, M, K, ldx, vp, mp, row_scale)
-                        : cudaLaunchKernelEx(&pc, prune_compress_fp8_kernel<false>, Xp, M, K, ldx, vp, mp, row_scale);
+    cudaError_t e;
+    if (row_amax)
+        e = (mode == LYNX_COMP_ROW)
+                ? cudaLaunchKernelEx(&pc, prune_compress_fp8_kernel<true, true>, Xp, M, K, ldx, row_amax, vp, mp, row_scale)
+                : cudaLaunchKernelEx(&pc, prune_compress_fp8_kernel<false, true>, Xp, M, K, ldx, row_amax, vp, mp, row_scale);
+    else
+        e = (mode == LYNX_COMP_ROW)
+                ? cudaLaunchKernelEx(&pc, prune_compress_fp8_kernel<true, false>, Xp, M, K, ldx, row_amax, vp, mp, row_scale)
+                : cudaLaunchKernelEx(&pc, prune_compress_fp8_kernel<false, false>, Xp, M, K, ldx, row_amax, vp, mp, row_scale);
     if (e != cudaSuccess) return LYNX_ERR_CUDA;
     ctx->launches++;
     return LYNX_OK;
@@ -1076,7 +1083,8 @@ lynx_status lynx_sparse_linear_fp8(lynx_ctx* ctx, const void* values_q, const vo
 }
 
 lynx_status lynx_act_sparse_linear_fp8(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx,
-                                       const void* Wq, int64_t N, int64_t ldwq, const float* wscale,
+                                       const float* row_amax, const void* Wq, int64_t N, int64_t ldwq,
+                                       const float* wscale,
                                        const void* bias, lynx_comp_mode mode, const void* residual, int64_t ldr,
                                        void* Y, int64_t ldy, void* stream) {
     lynx_status s = check_fp8_shape(ctx, M, K);
@@ -1099,7 +1107,7 @@ lynx_status lynx_act_sparse_linear_fp8(lynx_ctx* ctx, const void* X, int64_t M, 
     void* values_q = base + L.values;  // (sized for bf16 values: twice what the codes need)
     void* meta = base + L.meta;
     float* scale = reinterpret_cast<float*>(base + L.scale);
-    s = lynx_prune_compress_fp8(ctx, X, M, K, ldx, values_q, meta, scale, mode, stream);
+    s = lynx_prune_compress_fp8(ctx, X, M, K, ldx, row_amax, values_q, meta, scale, mode, stream);
     if (s != LYNX_OK) return s;
     lynx_comp comp;
     comp.row_scale = scale;

@@ -122,9 +122,10 @@ def main():
 
 
 def fp8_sweep(lx, shapes, iters):
-    print("| M | K | N | prune fp8 us | GEMM fp8 us | GEMM fp8 TF | layer fp8 us | layer bf16 us | dense bf16 us | "
-          "dense fp8 (torch) us | fp8 layer / bf16 layer | fp8 layer / dense bf16 | fp8 layer / dense fp8 |")
-    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+    print("| M | K | N | prune fp8 us | prune fp8 (given amax) us | GEMM fp8 us | GEMM fp8 TF | layer fp8 us | "
+          "layer fp8 (given amax) us | layer bf16 us | dense bf16 us | dense fp8 (torch) us | fp8 layer / bf16 layer | "
+          "fp8 layer / dense bf16 | fp8 layer / dense fp8 |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     for (M, K, N) in shapes:
         if K % 256:
             continue
@@ -142,6 +143,10 @@ def fp8_sweep(lx, shapes, iters):
         tg = timeloop(lambda j: lx.sparse_linear_fp8(cs[j][0], cs[j][1], Wqs[j][0], Wqs[j][1], b, cs[j][2], None, Ys[j]),
                       nsets, iters)
         tl = timeloop(lambda j: lx.act_sparse_linear_fp8(Xs[j], Wqs[j][0], Wqs[j][1], b, 1, None, Ys[j]), nsets, iters)
+        am = [X.float().abs().amax(dim=1).contiguous() for X in Xs]
+        tpg = timeloop(lambda j: lx.prune_compress_fp8(Xs[j], 1, *cs[j], row_amax=am[j]), nsets, iters)
+        tlg = timeloop(lambda j: lx.act_sparse_linear_fp8(Xs[j], Wqs[j][0], Wqs[j][1], b, 1, None, Ys[j], row_amax=am[j]),
+                       nsets, iters)
         tb = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_SEPARATE), nsets, iters)
         td = timeloop(lambda j: torch.nn.functional.linear(Xs[j], Ws[j], b), nsets, iters)
         # torch's dense FP8 GEMM (cuBLASLt) on pre-quantised operands, per-tensor scales
@@ -154,8 +159,9 @@ def fp8_sweep(lx, shapes, iters):
         except Exception:
             t8 = float("nan")
         fl = 2.0 * M * N * K
-        print(f"| {M} | {K} | {N} | {tp*1e3:.1f} | {tg*1e3:.1f} | {fl/tg/1e9:.0f} | {tl*1e3:.1f} | {tb*1e3:.1f} | "
-              f"{td*1e3:.1f} | {t8*1e3:.1f} | {tb/tl:.2f} | {td/tl:.2f} | {t8/tl:.2f} |", flush=True)
+        print(f"| {M} | {K} | {N} | {tp*1e3:.1f} | {tpg*1e3:.1f} | {tg*1e3:.1f} | {fl/tg/1e9:.0f} | {tl*1e3:.1f} | "
+              f"{tlg*1e3:.1f} | {tb*1e3:.1f} | {td*1e3:.1f} | {t8*1e3:.1f} | {tb/tl:.2f} | {td/tl:.2f} | {t8/tl:.2f} |",
+              flush=True)
         assert lx.last_error() == 0
         del Xs, Ws, Ys, Wqs, cs, Xq, Wt
         torch.cuda.empty_cache()

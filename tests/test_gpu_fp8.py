@@ -63,6 +63,37 @@ def test_activation_codes_metadata_and_scale(lx, M, K, dist, mode):
     np.testing.assert_allclose(rs.cpu().numpy(), ref_scale, rtol=1e-5)
 
 
+@pytest.mark.parametrize("M,K,mode", [(300, 1024, 1), (129, 256, 0), (2048, 3072, 1)])
+def test_supplied_row_maximum(lx, M, K, mode):
+    """The true maxima supplied by the caller give the same bits as the two-pass form; a
+    calibrated constant (some rows saturate, the rest lose range) matches the oracle."""
+    X = inputs.make_x(M, K, "outlier", 820 + M)
+    Xc = X.cuda()
+    vq, meta, rs = lx.prune_compress_fp8(Xc, mode)
+    amax = X.float().abs().max(dim=1).values
+    vq1, meta1, rs1 = lx.prune_compress_fp8(Xc, mode, row_amax=amax.cuda())
+    assert torch.equal(vq, vq1) and torch.equal(meta, meta1) and torch.equal(rs, rs1)
+    const = torch.full((M,), float(amax.median()), dtype=torch.float32)
+    vq2, meta2, rs2 = lx.prune_compress_fp8(Xc, mode, row_amax=const.cuda())
+    ov, om, oact = oracle.compress_fp8(u16(X), row_amax=const.numpy())
+    assert (vq2.cpu().numpy() == ov).all()
+    assert (meta2.cpu().numpy() == oracle.meta_canon_to_hw_fp8(om, M, K)).all()
+    ref = oracle.row_scale(u16(X), mode).astype(np.float64) * oact.astype(np.float64)
+    np.testing.assert_allclose(rs2.cpu().numpy(), ref, rtol=1e-5)
+    assert (np.abs(oracle.e4m3_decode(ov)) == 448.0).sum() > 0   # the constant does saturate some rows
+
+
+def test_layer_with_supplied_row_maximum(lx):
+    wl = inputs.WORKLOADS["tiny"]
+    d = inputs.make_workload(wl, with_bias=True)
+    amax = (d["X"].float().abs().max(dim=1).values * 1.25).contiguous()
+    oq, ows = oracle.quantize_weights_fp8(u16(d["W"]), True)
+    ref = oracle.act_sparse_linear_fp8(u16(d["X"]), oq, ows, bias=u16(d["bias"]), comp_mode=1, row_amax=amax.numpy())
+    Wq, ws = lx.quantize_weights_fp8(d["W"].cuda(), True)
+    Y = lx.act_sparse_linear_fp8(d["X"].cuda(), Wq, ws, d["bias"].cuda(), 1, row_amax=amax.cuda())
+    check_y(Y, ref["Y"])
+
+
 def test_activation_special_values(lx):
     M, K = 32, 256
     g = torch.Generator().manual_seed(5)
