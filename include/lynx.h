@@ -190,7 +190,10 @@ LYNX_API lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_
 /* Same layer with the activations and the result in HOST memory (pinned memory recommended):
  * X_host [M x K] and Y_host [M x N] are dense row-major bf16 HOST buffers; W and bias stay
  * DEVICE resident (weights are loaded once).  Copies X to the device, runs the layer, copies Y
- * back and synchronises `stream`.  Staging buffers live in the context's scratch. */
+ * back and synchronises `stream`.  Staging buffers live in the context's scratch.  From 2048 rows
+ * on (and not under LYNX_COMP_TENSOR, whose scale couples all rows) the call is pipelined over row
+ * chunks on two copy streams the context owns, so that copy-in, kernels and copy-out overlap; the
+ * result is the unchunked one bit for bit. */
 LYNX_API lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_host, int64_t M,
                                                  int64_t K, const void* W, int64_t N, int64_t ldw,
                                                  const void* bias, lynx_comp_mode mode, void* Y_host,

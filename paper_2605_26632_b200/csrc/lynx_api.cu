@@ -28,6 +28,9 @@ struct lynx_ctx {
     uint32_t* tickets = nullptr;  // one word per 16-row block (prune finalize), zero between launches
     void* lora_ws = nullptr;      // low-rank branch: [fp32 partials][T]
     size_t lora_ws_bytes = 0;
+    // host-buffer entry point: copy streams and events of its row-chunk pipeline (created on first use)
+    cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+    cudaEvent_t ev_h2d[8] = {}, ev_done[8] = {}, ev_all = nullptr;
     uint32_t l0_epoch = 0;        // launch counter of the fused down projection (ready words hold it)
     uint32_t l0_done_total = 0;   // groups published by all such launches so far (mod 2^32)
     int l0_force_splits = 0, l0_force_fill = -1;  // development overrides of the phase-0 plan
@@ -665,6 +668,13 @@ lynx_status lynx_destroy(lynx_ctx* ctx) {
     if (ctx->sk_partial) cudaFree(ctx->sk_partial);
     if (ctx->tickets) cudaFree(ctx->tickets);
     if (ctx->lora_ws) cudaFree(ctx->lora_ws);
+    if (ctx->h2d_stream) cudaStreamDestroy(ctx->h2d_stream);
+    if (ctx->d2h_stream) cudaStreamDestroy(ctx->d2h_stream);
+    for (int i = 0; i < 8; ++i) {
+        if (ctx->ev_h2d[i]) cudaEventDestroy(ctx->ev_h2d[i]);
+        if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
+    }
+    if (ctx->ev_all) cudaEventDestroy(ctx->ev_all);
     if (ctx->err_host) cudaFreeHost(ctx->err_host);
     delete ctx;
     return LYNX_OK;
@@ -880,15 +890,61 @@ lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_host, int64
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(ctx->scratch);
-    void* xd = base + L.xstage;
-    void* yd = base + L.ystage;
-    if (cudaMemcpyAsync(xd, X_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    char* xd = base + L.xstage;
+    char* yd = base + L.ystage;
+    // Token rows are independent (except under the whole-tensor scale), so the call is pipelined over
+    // row chunks: the copy-in of chunk c + 1 and the copy-out of chunk c - 1 overlap the kernels of
+    // chunk c on two copy streams (PCIe is full duplex); the result is the unchunked one bit for bit.
+    int chunks = (M >= 2048 && mode != LYNX_COMP_TENSOR) ? 4 : 1;
+    const int64_t rows_per = ((M + chunks - 1) / chunks + 255) / 256 * 256;
+    chunks = (int)((M + rows_per - 1) / rows_per);
+    if (chunks == 1) {
+        if (cudaMemcpyAsync(xd, X_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return LYNX_ERR_CUDA;
+        s = lynx_act_sparse_linear(ctx, xd, M, K, K, W, N, ldw, bias, mode, nullptr, 0, yd, N, fuse, stream);
+        if (s != LYNX_OK) return s;
+        if (cudaMemcpyAsync(Y_host, yd, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return LYNX_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return LYNX_ERR_CUDA;
+        return check_device_error(ctx);
+    }
+    if (!ctx->h2d_stream) {
+        std::lock_guard<std::mutex> lock(ctx->mu);
+        bool ok = cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&ctx->ev_all, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < 8 && ok; ++i)
+            ok = cudaEventCreateWithFlags(&ctx->ev_h2d[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return LYNX_ERR_CUDA;
+    }
+    // the copy streams start behind whatever the caller already queued on `stream`
+    if (cudaEventRecord(ctx->ev_all, st) != cudaSuccess || cudaStreamWaitEvent(ctx->h2d_stream, ctx->ev_all, 0) != cudaSuccess)
         return LYNX_ERR_CUDA;
-    s = lynx_act_sparse_linear(ctx, xd, M, K, K, W, N, ldw, bias, mode, nullptr, 0, yd, N, fuse, stream);
-    if (s != LYNX_OK) return s;
-    if (cudaMemcpyAsync(Y_host, yd, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    const char* xh = static_cast<const char*>(X_host);
+    char* yh = static_cast<char*>(Y_host);
+    for (int c = 0; c < chunks; ++c) {
+        const int64_t r0 = c * rows_per, rows = (r0 + rows_per <= M) ? rows_per : M - r0;
+        if (cudaMemcpyAsync(xd + (size_t)r0 * K * 2, xh + (size_t)r0 * K * 2, (size_t)rows * K * 2,
+                            cudaMemcpyHostToDevice, ctx->h2d_stream) != cudaSuccess ||
+            cudaEventRecord(ctx->ev_h2d[c], ctx->h2d_stream) != cudaSuccess)
+            return LYNX_ERR_CUDA;
+    }
+    for (int c = 0; c < chunks; ++c) {
+        const int64_t r0 = c * rows_per, rows = (r0 + rows_per <= M) ? rows_per : M - r0;
+        if (cudaStreamWaitEvent(st, ctx->ev_h2d[c], 0) != cudaSuccess) return LYNX_ERR_CUDA;
+        s = lynx_act_sparse_linear(ctx, xd + (size_t)r0 * K * 2, rows, K, K, W, N, ldw, bias, mode, nullptr, 0,
+                                   yd + (size_t)r0 * N * 2, N, fuse, stream);
+        if (s != LYNX_OK) return s;
+        if (cudaEventRecord(ctx->ev_done[c], st) != cudaSuccess ||
+            cudaStreamWaitEvent(ctx->d2h_stream, ctx->ev_done[c], 0) != cudaSuccess ||
+            cudaMemcpyAsync(yh + (size_t)r0 * N * 2, yd + (size_t)r0 * N * 2, (size_t)rows * N * 2,
+                            cudaMemcpyDeviceToHost, ctx->d2h_stream) != cudaSuccess)
+            return LYNX_ERR_CUDA;
+    }
+    if (cudaEventRecord(ctx->ev_all, ctx->d2h_stream) != cudaSuccess || cudaStreamWaitEvent(st, ctx->ev_all, 0) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
         return LYNX_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return LYNX_ERR_CUDA;
     return check_device_error(ctx);
 }
 

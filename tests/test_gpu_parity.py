@@ -264,6 +264,20 @@ def test_host_buffer_entry_point(lx):
     check_y(Y, ref["Y"])
 
 
+@pytest.mark.parametrize("M,mode", [(2500, 1), (4096, 0), (2304, 2)])
+def test_host_buffer_entry_point_pipelined_chunks(lx, M, mode):
+    """From 2048 rows on the host entry point pipelines row chunks over copy streams (not under the
+    whole-tensor scale): same bits as the device-buffer call, twice in a row."""
+    K, N = 512, 776
+    X = inputs.make_x(M, K, "outlier", 61)
+    W, b = inputs.make_w(N, K, 61).cuda(), inputs.make_bias(N, 61).cuda()
+    want = lx.act_sparse_linear(X.cuda(), W, b, mode).cpu()
+    Xh = X.pin_memory()
+    for _ in range(2):
+        Y = lx.act_sparse_linear_host(Xh, W, b, mode)
+        assert torch.equal(Y, want)
+
+
 # ------------------------------------------------------------------ fused one-kernel path ------
 
 @pytest.mark.parametrize("mode", [0, 1])
