@@ -219,6 +219,24 @@ def test_ragged_shapes(lx, M, K, N):
     check_y(Y, ref["Y"])
 
 
+def test_leading_dimensions_of_w_y_and_residual(lx):
+    """W, Y and the residual as column slices of wider buffers (ld > extent); nothing outside the
+    Y slice may be written."""
+    M, K, N = 300, 384, 456
+    X = inputs.make_x(M, K, "outlier", 91)
+    Wbig = torch.zeros(N, K + 128, dtype=torch.bfloat16)
+    Wbig[:, :K] = inputs.make_w(N, K, 91)
+    Rbig = torch.zeros(M, N + 64, dtype=torch.bfloat16)
+    Rbig[:, :N] = inputs.make_residual(M, N, 91)
+    b = inputs.make_bias(N, 91)
+    ref = oracle.act_sparse_linear(u16(X), u16(Wbig[:, :K].contiguous()), bias=u16(b), comp_mode=1,
+                                   Yr=u16(Rbig[:, :N].contiguous()))
+    Ybig = torch.full((M, N + 72), 3.0, dtype=torch.bfloat16, device="cuda")
+    Y = lx.act_sparse_linear(X.cuda(), Wbig.cuda()[:, :K], b.cuda(), 1, Rbig.cuda()[:, :N], out=Ybig[:, :N])
+    check_y(Y, ref["Y"])
+    assert (Ybig[:, N:] == 3.0).all()
+
+
 def test_integer_valued_inputs_are_exact(lx):
     """Small integers: every partial sum is exact in fp32 and in bf16, so Y must equal the oracle."""
     rng = np.random.default_rng(4)
