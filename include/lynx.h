@@ -23,6 +23,8 @@
  *   - Shape rules: M >= 1, K % 128 == 0, N % 8 == 0; base pointers and leading dimensions must be
  *     16-byte aligned (ld % 8 == 0 for bf16).  Row tails (M not a multiple of the tile) are
  *     handled inside the kernels.
+ *   - A context belongs to one device, and that device must be the calling thread's current
+ *     device (cudaSetDevice) whenever the context is used; lynx_create makes it current.
  *   - There is no CPU fallback: on a device that is not sm_100 lynx_create fails with
  *     LYNX_ERR_UNSUPPORTED_ARCH.
  */

@@ -82,6 +82,18 @@ bool make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const 
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// cudaFuncSetAttribute is per device: remember, per kernel instantiation, which devices have it.
+constexpr int MAX_CTX_DEVICES = 64;
+template <class Kernel>
+lynx_status allow_dynamic_smem(Kernel kern, int bytes, int device, bool (&done)[MAX_CTX_DEVICES]) {
+    if (device < 0 || device >= MAX_CTX_DEVICES) return LYNX_ERR_INVALID_ARG;
+    if (done[device]) return LYNX_OK;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+        return LYNX_ERR_CUDA;
+    done[device] = true;
+    return LYNX_OK;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 lynx_status check_device_error(lynx_ctx* ctx) {
@@ -261,12 +273,9 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     p.ldt = 0;
 
     auto kern = lora ? sparse_gemm_kernel<Cfg, true> : sparse_gemm_kernel<Cfg, false>;
-    static bool attr_set[2] = {false, false};  // per instantiation
-    if (!attr_set[lora ? 1 : 0]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-            return LYNX_ERR_CUDA;
-        attr_set[lora ? 1 : 0] = true;
-    }
+    static bool attr_set[2][MAX_CTX_DEVICES] = {};  // per instantiation (with / without the low-rank code)
+    if (lynx_status as = allow_dynamic_smem(kern, Cfg::SMEM_BYTES, ctx->device, attr_set[lora ? 1 : 0]); as != LYNX_OK)
+        return as;
     const int tiles = p.tiles_m * p.tiles_n;
     int clusters = ctx->num_sms / Cfg::CG;
     {
@@ -404,12 +413,8 @@ lynx_status launch_gemm_fp8_cfg(lynx_ctx* ctx, const void* values_q, const void*
     p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
     p.l0_splits = 1;
     auto kern = sparse_gemm_kernel<Cfg, false>;
-    static bool attr_set = false;  // per instantiation
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-            return LYNX_ERR_CUDA;
-        attr_set = true;
-    }
+    static bool attr_set[MAX_CTX_DEVICES] = {};  // per instantiation
+    if (lynx_status as = allow_dynamic_smem(kern, Cfg::SMEM_BYTES, ctx->device, attr_set); as != LYNX_OK) return as;
     const int tiles = p.tiles_m * p.tiles_n;
     int clusters = ctx->num_sms / Cfg::CG;
     if (clusters > tiles) clusters = tiles;
@@ -473,13 +478,9 @@ lynx_status launch_fused(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int
     p.dev_error = ctx->err_dev;
     p.tiles_m = (int)((M + Cfg::BM - 1) / Cfg::BM);
     p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(fused_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Cfg::SMEM_BYTES) != cudaSuccess)
-            return LYNX_ERR_CUDA;
-        attr_set = true;
-    }
+    static bool attr_set[MAX_CTX_DEVICES] = {};
+    if (lynx_status as = allow_dynamic_smem(fused_linear_kernel, Cfg::SMEM_BYTES, ctx->device, attr_set); as != LYNX_OK)
+        return as;
     int grid = p.tiles_m * p.tiles_n;
     if (grid > ctx->num_sms) grid = ctx->num_sms;
     fused_linear_kernel<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, st>>>(tx, tb, ty, p);
@@ -581,12 +582,8 @@ lynx_status launch_lora_down(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
     p.tickets = ctx->tickets + PRUNE_TICKET_BYTES / 4;
     p.dev_error = ctx->err_dev;
     auto kern = lora_down_kernel<Cfg>;
-    static bool attr_set = false;  // per instantiation
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-            return LYNX_ERR_CUDA;
-        attr_set = true;
-    }
+    static bool attr_set[MAX_CTX_DEVICES] = {};  // per instantiation
+    if (lynx_status as = allow_dynamic_smem(kern, Cfg::SMEM_BYTES, ctx->device, attr_set); as != LYNX_OK) return as;
     const int tiles_m = (int)((M + Cfg::BM - 1) / Cfg::BM);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(tiles_m * p.splits));
