@@ -267,13 +267,19 @@ def main():
         j = i % NSETS
         lx.act_sparse_linear(Xs[j], Ws[j], bias, comp_mode, None, Ys[j], binding.FUSE_SEPARATE)
 
+    def probe_scale(j):
+        # ROW mode: the deferred form, i.e. exactly the two launches the layer call makes
+        if comp_mode == 1:
+            return binding.ROW_SCALE_DEFERRED
+        return scales[j] if comp_mode else None
+
     def probe_step(i, ev):
         # the same two kernels as separate calls with an event between them (per-kernel times)
         j = i % NSETS
         ev[0].record(stream)
-        lx.prune_compress(Xs[j], comp_mode, vals[j], metas[j], scales[j] if comp_mode else None)
+        lx.prune_compress(Xs[j], comp_mode, vals[j], metas[j], probe_scale(j))
         ev[1].record(stream)
-        lx.sparse_linear(vals[j], metas[j], Ws[j], bias, scales[j] if comp_mode else None, None, Ys[j])
+        lx.sparse_linear(vals[j], metas[j], Ws[j], bias, probe_scale(j), None, Ys[j])
         ev[2].record(stream)
 
     def barrier():
@@ -305,8 +311,8 @@ def main():
 
     # per-kernel times: the same number of steps again, as two calls with CUDA events around each
     # kernel (an event between two launches keeps the second kernel from starting early as a
-    # programmatic dependent, and the stand-alone prune call finalizes the row scale itself instead
-    # of leaving the sums to the GEMM epilogue, so these steps are a little slower than the timed ones)
+    # programmatic dependent, so these steps are a little slower than the timed ones; in ROW mode the
+    # two calls use the deferred row scale, i.e. they are the launches the layer call makes)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     probed = list(range(args.steps))
     for i in probed:
@@ -318,17 +324,23 @@ def main():
 
     # prune/compress (row scale finalized in the same launch) alone, back to back over the rotating sets: the
     # per-launch time that the HBM roofline of that kernel is computed from
-    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for i in range(3):
-        lx.prune_compress(Xs[i % NSETS], comp_mode, vals[i % NSETS], metas[i % NSETS], scales[i % NSETS] if comp_mode else None)
-    torch.cuda.synchronize()
-    p0.record(stream)
-    for i in range(args.steps):
-        j = i % NSETS
-        lx.prune_compress(Xs[j], comp_mode, vals[j], metas[j], scales[j] if comp_mode else None)
-    p1.record(stream)
-    torch.cuda.synchronize()
-    prune_loop_ms = p0.elapsed_time(p1) / args.steps
+    def prune_loop(scale_of):
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(3):
+            lx.prune_compress(Xs[i % NSETS], comp_mode, vals[i % NSETS], metas[i % NSETS], scale_of(i % NSETS))
+        torch.cuda.synchronize()
+        p0.record(stream)
+        for i in range(args.steps):
+            j = i % NSETS
+            lx.prune_compress(Xs[j], comp_mode, vals[j], metas[j], scale_of(j))
+        p1.record(stream)
+        torch.cuda.synchronize()
+        return p0.elapsed_time(p1) / args.steps
+
+    # as launched by the layer call (ROW mode: the scale is finished by the GEMM epilogue), and the
+    # stand-alone form that finishes the scale in the same launch
+    prune_loop_ms = prune_loop(probe_scale)
+    prune_alone_ms = prune_loop(lambda j: scales[j] if comp_mode else None)
 
     # dense bf16 GEMM of the same shape on the same GPU (same rotation, same event timing)
     dense_out = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
@@ -433,8 +445,12 @@ def main():
         "roofline_prune": {"bound": "hbm", "kernel": "prune_compress_kernel", "achieved": prune_gbs,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": prune_gbs / peaks["hbm_gbs"],
                            "frac_of_8TBs_nominal": prune_gbs / 8000.0, "bytes_per_launch": prune_bytes, "ms_per_launch": prune_loop_ms,
-                           "how": "back-to-back loop of lynx_prune_compress (one launch: select, compress, row sums, scale) over "
-                                  "rotating buffers, CUDA events; the in-step figure is kernels.prune_compress_ms",
+                           "standalone_ms_per_launch": prune_alone_ms,
+                           "standalone_frac": prune_bytes / (prune_alone_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                           "how": "back-to-back loop of lynx_prune_compress over rotating buffers, CUDA events: the form the "
+                                  "layer call launches (select, compress, row sums; the GEMM epilogue finishes the scale) and, "
+                                  "as standalone_*, the form that also finishes the scale in the same launch; the in-step "
+                                  "figure is kernels.prune_compress_ms",
                            "peak_kind": f"hbm_gbs ({peaks['source']})"},
         "clocks": clocks,
         "e2e": e2e,

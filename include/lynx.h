@@ -72,9 +72,18 @@ typedef enum {
     LYNX_FUSE_FUSED = 2     /* one kernel, compressed activations never written to HBM        */
 } lynx_fuse_mode;
 
+/* "Deferred" row scale for the two-call form (what lynx_act_sparse_linear does internally in
+ * LYNX_COMP_ROW mode): pass this value as `row_scale` to lynx_prune_compress and the kernel stops
+ * at its per-K-split row sums, kept in the context, instead of finishing s_m itself (which costs a
+ * hand-over between its CTAs); pass it as comp->row_scale to the lynx_sparse_linear call that
+ * follows ON THE SAME CONTEXT with the same M and K, and its epilogue forms s_m from those sums,
+ * in the same order of additions (same bits).  A later lynx_prune_compress or layer call on the
+ * context overwrites the sums. */
+#define LYNX_ROW_SCALE_DEFERRED ((float*)(uintptr_t)1)
+
 /* Epilogue terms of lynx_sparse_linear (all optional). */
 typedef struct {
-    const float* row_scale; /* [M] fp32 per-row scale s_m, or NULL (= 1)                      */
+    const float* row_scale; /* [M] fp32 per-row scale s_m, NULL (= 1), or LYNX_ROW_SCALE_DEFERRED  */
     const void* residual;   /* Y_r: [M x N] bf16, leading dimension ldr, or NULL              */
     int64_t ldr;
 } lynx_comp;

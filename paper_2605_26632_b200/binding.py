@@ -28,6 +28,18 @@ EXPORTS = [
 ]
 
 
+class _Deferred:
+    """Pass as ``row_scale`` to ``Lynx.prune_compress`` (ROW mode) and to the ``Lynx.sparse_linear`` call
+    that follows on the same context: the prune kernel stops at its row sums and the GEMM epilogue
+    forms the scale from them (``LYNX_ROW_SCALE_DEFERRED``)."""
+
+    def __repr__(self):
+        return "ROW_SCALE_DEFERRED"
+
+
+ROW_SCALE_DEFERRED = _Deferred()
+
+
 class LynxError(RuntimeError):
     def __init__(self, status: int, what: str):
         super().__init__(f"{what}: lynx status {status} ({status_string(status)})")
@@ -191,8 +203,9 @@ class Lynx:
             meta = torch.empty(meta_bytes(M, K), dtype=torch.uint8, device=X.device)
         if row_scale is None and mode in (COMP_ROW, COMP_TENSOR):
             row_scale = torch.empty(M, dtype=torch.float32, device=X.device)
+        rs = ctypes.c_void_p(1) if row_scale is ROW_SCALE_DEFERRED else _ptr(row_scale)
         _check(self._lib.lynx_prune_compress(self._h, _ptr(X), M, K, X.stride(0), _ptr(values), _ptr(meta),
-                                             _ptr(row_scale), mode, _stream()), "lynx_prune_compress")
+                                             rs, mode, _stream()), "lynx_prune_compress")
         return values, meta, row_scale
 
     def sparse_linear(self, values: torch.Tensor, meta: torch.Tensor, W: torch.Tensor, bias=None,
@@ -203,7 +216,7 @@ class Lynx:
         N = W.shape[0]
         if out is None:
             out = torch.empty((M, N), dtype=torch.bfloat16, device=values.device)
-        comp = _Comp(None if row_scale is None else row_scale.data_ptr(),
+        comp = _Comp(1 if row_scale is ROW_SCALE_DEFERRED else (None if row_scale is None else row_scale.data_ptr()),
                      None if residual is None else residual.data_ptr(),
                      0 if residual is None else residual.stride(0))
         _check(self._lib.lynx_sparse_linear(self._h, _ptr(values), _ptr(meta), M, K, _ptr(W), N, W.stride(0),

@@ -31,6 +31,10 @@ struct lynx_ctx {
     // host-buffer entry point: copy streams and events of its row-chunk pipeline (created on first use)
     cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
     cudaEvent_t ev_h2d[8] = {}, ev_done[8] = {}, ev_all = nullptr;
+    // row sums the last deferred prune launch left in the scratch (two-call form), and their shape
+    const float* deferred_partial = nullptr;
+    int deferred_ks = 0;
+    int64_t deferred_M = 0, deferred_K = 0;
     uint32_t l0_epoch = 0;        // launch counter of the fused down projection (ready words hold it)
     uint32_t l0_done_total = 0;   // groups published by all such launches so far (mod 2^32)
     int l0_force_splits = 0, l0_force_fill = -1;  // development overrides of the phase-0 plan
@@ -793,11 +797,21 @@ static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
         src->partial = defer ? partial : nullptr;
         src->ks = defer ? KS : 0;
     }
+    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_GROUP) {  // the scratch's sums now belong to this call
+        ctx->deferred_partial = defer ? partial : nullptr;
+        ctx->deferred_ks = defer ? KS : 0;
+        ctx->deferred_M = M;
+        ctx->deferred_K = K;
+    }
     return cuda_ok(cudaGetLastError());
 }
 
 lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, void* values,
                                 void* meta, float* row_scale, lynx_comp_mode mode, void* stream) {
+    if (row_scale == LYNX_ROW_SCALE_DEFERRED) {
+        if (mode != LYNX_COMP_ROW) return LYNX_ERR_INVALID_ARG;
+        return prune_impl(ctx, X, M, K, ldx, values, meta, nullptr, mode, stream, true, nullptr);
+    }
     return prune_impl(ctx, X, M, K, ldx, values, meta, row_scale, mode, stream, false, nullptr);
 }
 
@@ -817,6 +831,17 @@ lynx_status lynx_sparse_linear(lynx_ctx* ctx, const void* values, const void* me
         if (!aligned16(comp->residual) || (comp->ldr % 8)) return LYNX_ERR_ALIGNMENT;
     }
     if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+    if (comp && comp->row_scale == LYNX_ROW_SCALE_DEFERRED) {
+        // the sums of the deferred prune call that preceded this one on the context
+        if (!ctx->deferred_partial || ctx->deferred_M != M || ctx->deferred_K != K) return LYNX_ERR_INVALID_ARG;
+        ScaleSrc ss;
+        ss.partial = ctx->deferred_partial;
+        ss.ks = ctx->deferred_ks;
+        lynx_comp c2 = *comp;
+        c2.row_scale = nullptr;
+        return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &c2, nullptr, Y, ldy,
+                           static_cast<cudaStream_t>(stream), 0, &ss);
+    }
     return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, comp, nullptr, Y, ldy,
                        static_cast<cudaStream_t>(stream));
 }
@@ -958,7 +983,7 @@ lynx_status lynx_lora_down(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, i
     lynx_status s = check_common(ctx, M, K);
     if (s != LYNX_OK) return s;
     if ((s = check_lora_rank(R)) != LYNX_OK) return s;
-    if (!X || !LB || !T) return LYNX_ERR_INVALID_ARG;
+    if (!X || !LB || !T || row_scale == LYNX_ROW_SCALE_DEFERRED) return LYNX_ERR_INVALID_ARG;
     if (ldx < K || ldlb < K || ldt < R) return LYNX_ERR_INVALID_ARG;
     if ((size_t)((M + 127) / 128) * 4 > LORA_TICKET_BYTES) return LYNX_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(X) || !aligned16(LB) || !aligned16(T) || (ldx % 8) || (ldlb % 8) || (ldt % 8))
@@ -983,6 +1008,7 @@ lynx_status lynx_sparse_linear_lora(lynx_ctx* ctx, const void* values, const voi
     if (s != LYNX_OK) return s;
     if ((s = check_lora_rank(R)) != LYNX_OK) return s;
     if (!values || !meta || !W || !Y || !T || !LA || N < 8) return LYNX_ERR_INVALID_ARG;
+    if (comp && comp->row_scale == LYNX_ROW_SCALE_DEFERRED) return LYNX_ERR_INVALID_ARG;  // T needs the finished scale
     if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
     if (ldw < K || ldy < N || ldt < R || ldla < R) return LYNX_ERR_INVALID_ARG;
     if (!aligned16(values) || !aligned16(meta) || !aligned16(W) || !aligned16(Y) || !aligned16(T) || !aligned16(LA) ||
@@ -1121,6 +1147,7 @@ lynx_status lynx_sparse_linear_fp8(lynx_ctx* ctx, const void* values_q, const vo
     lynx_status s = check_fp8_shape(ctx, M, K);
     if (s != LYNX_OK) return s;
     if (!values_q || !meta || !Wq || !Y || N < 8) return LYNX_ERR_INVALID_ARG;
+    if (comp && comp->row_scale == LYNX_ROW_SCALE_DEFERRED) return LYNX_ERR_INVALID_ARG;
     if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
     if (ldwq < K || ldy < N) return LYNX_ERR_INVALID_ARG;
     if (!aligned16(values_q) || !aligned16(meta) || !aligned16(Wq) || !aligned16(Y) || (ldwq % 16) || (ldy % 8))

@@ -237,6 +237,31 @@ def test_leading_dimensions_of_w_y_and_residual(lx):
     assert (Ybig[:, N:] == 3.0).all()
 
 
+def test_deferred_row_scale_two_call_form(lx):
+    """The prune call stops at its row sums, the GEMM epilogue finishes the scale: same bits as
+    the form that finishes the scale inside the prune kernel, and as the layer call."""
+    from paper_2605_26632_b200 import binding
+    from paper_2605_26632_b200.binding import LynxError
+
+    M, K, N = 700, 1664, 1096
+    X = inputs.make_x(M, K, "outlier", 33).cuda()
+    W, b = inputs.make_w(N, K, 33).cuda(), inputs.make_bias(N, 33).cuda()
+    v, m, s = lx.prune_compress(X, 1)
+    want = lx.sparse_linear(v, m, W, b, s)
+    v2, m2, d = lx.prune_compress(X, 1, row_scale=binding.ROW_SCALE_DEFERRED)
+    assert d is binding.ROW_SCALE_DEFERRED and torch.equal(v, v2) and torch.equal(m, m2)
+    got = lx.sparse_linear(v2, m2, W, b, binding.ROW_SCALE_DEFERRED)
+    assert torch.equal(got, want)
+    assert torch.equal(lx.act_sparse_linear(X, W, b, 1), want)
+    # the sums belong to the last prune call of that shape: another shape is refused, nothing is launched
+    X2 = inputs.make_x(256, 512, "gelu", 1).cuda()
+    v3, m3, _ = lx.prune_compress(X2, 1, row_scale=binding.ROW_SCALE_DEFERRED)
+    n0 = lx.launch_count()
+    with pytest.raises(LynxError) as e:
+        lx.sparse_linear(v2, m2, W, b, binding.ROW_SCALE_DEFERRED)
+    assert e.value.status == 1 and lx.launch_count() == n0
+
+
 def test_integer_valued_inputs_are_exact(lx):
     """Small integers: every partial sum is exact in fp32 and in bf16, so Y must equal the oracle."""
     rng = np.random.default_rng(4)
