@@ -278,9 +278,10 @@ LYNX_API lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, i
  * group g = (k % 128) / 4 in bits 4 * (g % 2) of byte g / 2; rows past M hold 0x4 nibbles.
  * row_amax (optional, [M] fp32 on the device): when given, row_amax[m] takes the place of the
  * row maximum found in the data -- a scale calibrated beforehand (the same number in every entry)
- * or a maximum the producer of X already knows; values beyond it saturate at +-448.  Without it
- * lynx_prune_compress_fp8 reads X twice (row maxima first; the second pass normally hits the L2),
- * with it once.  Neither form needs scratch.  The low-rank branch, LYNX_COMP_TENSOR / GROUP and the one-kernel mode are
+ * or a maximum the producer of X already knows; values beyond it saturate at +-448.  Either
+ * way X is read from device memory once for 2048 <= K <= ~57000 (whole rows are staged in shared
+ * memory: the maximum and the codes come from the staged copy); shorter and longer rows take a
+ * kernel that, without row_amax, reads them twice.  Neither form needs scratch.  The low-rank branch, LYNX_COMP_TENSOR / GROUP and the one-kernel mode are
  * not available in FP8.
  */
 LYNX_API lynx_status lynx_quantize_weights_fp8(lynx_ctx* ctx, const void* W, int64_t N, int64_t K,

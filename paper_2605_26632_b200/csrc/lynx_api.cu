@@ -48,6 +48,8 @@ struct lynx_ctx {
     int pdl = 1;        // programmatic dependent launch of the finalize and GEMM kernels
     int gemm_cfg = 0;   // 0 = auto
     int prune_tpu = 0;  // 0 = auto
+    int fp8_ring = 1;   // FP8 activations: single-read ring kernel (LYNX_FP8_RING=0: one CTA per 16 rows)
+    int fp8_ring_forced = 0;
     std::mutex mu;
 };
 
@@ -658,6 +660,11 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
     if (env) ctx->defer_scale = atoi(env);
     env = getenv("LYNX_PRUNE_TPU");  // development override: 128-element K blocks per warp
     if (env) ctx->prune_tpu = atoi(env);
+    env = getenv("LYNX_FP8_RING");  // development override: 0 = one CTA per 16 rows, n = ring with n warps per row
+    if (env) {
+        ctx->fp8_ring = atoi(env);
+        ctx->fp8_ring_forced = 1;
+    }
     *out = ctx;
     return LYNX_OK;
 }
@@ -1086,6 +1093,14 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
 
 // ------------------------------------------------------------------------- FP8 composition ------
 
+// Warps that share a row in the FP8 ring kernel: the fewest for which every group still gets a
+// slot of its own (all 16 consumer warps stay busy; longer rows are split over more warps).
+static int fp8_ring_group_width(int slots) {
+    int gw = 1;
+    while (gw < 8 && FP8_RING_CW / gw > slots) gw *= 2;
+    return gw;
+}
+
 static lynx_status check_fp8_shape(lynx_ctx* ctx, int64_t M, int64_t K) {
     lynx_status s = check_common(ctx, M, K);
     if (s != LYNX_OK) return s;
@@ -1128,6 +1143,40 @@ lynx_status lynx_prune_compress_fp8(lynx_ctx* ctx, const void* X, int64_t M, int
     uint8_t* vp = static_cast<uint8_t*>(values_q);
     uint8_t* mp = static_cast<uint8_t*>(meta);
     cudaError_t e;
+    // The persistent ring kernel reads X once (also when the maxima have to be found in the data).
+    // It wants at least two rows in shared memory and rows long enough to occupy a warp.
+    int slots = (int)((FP8_RING_SMEM_MAX - FP8_RING_HEADER) / (K * 2));
+    if (slots > FP8_RING_MAX_SLOTS) slots = FP8_RING_MAX_SLOTS;
+    if (ctx->fp8_ring && slots >= 2 && K >= 2048) {
+        // gw warps share a row; ng = CW / gw groups, each with at least one slot of its own
+        int gw = fp8_ring_group_width(slots);
+        if (ctx->fp8_ring_forced && (ctx->fp8_ring == 1 || ctx->fp8_ring == 2 || ctx->fp8_ring == 4 || ctx->fp8_ring == 8))
+            gw = ctx->fp8_ring;
+        int ng = FP8_RING_CW / gw;
+        if (ng > slots) ng = slots;
+        const int smem = FP8_RING_HEADER + slots * (int)(K * 2);
+        const bool sums = mode == LYNX_COMP_ROW, given = row_amax != nullptr;
+        using RingKernel = void (*)(const uint16_t*, int64_t, int64_t, int64_t, const float*, uint8_t*, uint8_t*,
+                                    float*, int, int, uint32_t*);
+#define LYNX_RING4(S, G) prune_compress_fp8_ring_kernel<S, G, 1>, prune_compress_fp8_ring_kernel<S, G, 2>, \
+                         prune_compress_fp8_ring_kernel<S, G, 4>, prune_compress_fp8_ring_kernel<S, G, 8>
+        static const RingKernel kerns[16] = {LYNX_RING4(false, false), LYNX_RING4(true, false),
+                                             LYNX_RING4(false, true), LYNX_RING4(true, true)};
+#undef LYNX_RING4
+        static bool attr_set[16][MAX_CTX_DEVICES] = {};
+        const int which = (sums ? 4 : 0) + (given ? 8 : 0) + (gw == 1 ? 0 : gw == 2 ? 1 : gw == 4 ? 2 : 3);
+        if (lynx_status as = allow_dynamic_smem(kerns[which], FP8_RING_SMEM_MAX, ctx->device, attr_set[which]);
+            as != LYNX_OK)
+            return as;
+        pc.gridDim = dim3((unsigned)(M < ctx->num_sms ? M : ctx->num_sms));
+        pc.blockDim = dim3(FP8_RING_THREADS);
+        pc.dynamicSmemBytes = (size_t)smem;
+        e = cudaLaunchKernelEx(&pc, kerns[which], Xp, M, K, ldx, row_amax, vp, mp, row_scale, slots, ng,
+                               ctx->err_dev);
+        if (e != cudaSuccess) return LYNX_ERR_CUDA;
+        ctx->launches++;
+        return LYNX_OK;
+    }
     if (row_amax)
         e = (mode == LYNX_COMP_ROW)
                 ? cudaLaunchKernelEx(&pc, prune_compress_fp8_kernel<true, true>, Xp, M, K, ldx, row_amax, vp, mp, row_scale)

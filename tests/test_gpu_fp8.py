@@ -63,6 +63,82 @@ def test_activation_codes_metadata_and_scale(lx, M, K, dist, mode):
     np.testing.assert_allclose(rs.cpu().numpy(), ref_scale, rtol=1e-5)
 
 
+# The single-read kernel (K >= 2048) splits a row over 1, 2, 4 or 8 warps depending on how many rows
+# fit in shared memory; the shapes below reach each split, a ragged last 128-row block, fewer rows
+# than SMs, a row range per CTA of uneven length, and a leading dimension larger than K.
+RING_SHAPES = [(300, 2048, 1), (77, 6144, 1), (1, 2048, 0), (513, 8192, 1), (200, 12288, 0), (130, 24576, 1),
+               (40, 49152, 1), (1000, 3072, 0)]
+
+
+@pytest.mark.parametrize("M,K,mode", RING_SHAPES)
+def test_single_read_kernel_shapes(lx, M, K, mode):
+    X = inputs.make_x(M, K, "outlier" if M % 2 else "gelu_chan", 900 + M)
+    ov, om, oact = oracle.compress_fp8(u16(X))
+    ref_scale = oracle.row_scale(u16(X), mode).astype(np.float64) * oact.astype(np.float64)
+    ometa = oracle.meta_canon_to_hw_fp8(om, M, K)
+    amax = X.float().abs().max(dim=1).values.contiguous().cuda()
+    for given in (None, amax):
+        vq, meta, rs = lx.prune_compress_fp8(X.cuda(), mode, row_amax=given)
+        assert (vq.cpu().numpy() == ov).all(), "codes differ"
+        assert (meta.cpu().numpy() == ometa).all(), "metadata differs"
+        np.testing.assert_allclose(rs.cpu().numpy(), ref_scale, rtol=1e-5)
+    # rows of a wider matrix (leading dimension 3 * 16 elements beyond K)
+    wide = torch.zeros((M, K + 48), dtype=torch.bfloat16)
+    wide[:, :K] = X
+    vq2, meta2, rs2 = lx.prune_compress_fp8(wide.cuda()[:, :K], mode)
+    assert torch.equal(vq2, vq) and torch.equal(meta2, meta) and torch.equal(rs2, rs)
+
+
+def test_single_read_kernel_special_values(lx):
+    """Zero rows, subnormals, infinities and NaN through the shared-memory path (K = 2048)."""
+    M, K = 40, 2048
+    g = torch.Generator().manual_seed(6)
+    x = torch.randn(M, K, generator=g)
+    x[0] = 0.0
+    x[1, 0:4] = torch.tensor([1e-40, -1e-40, 2e-40, 0.0])
+    x[2, 1037] = float("inf")
+    x[3, 2047] = float("nan")
+    x[5, 100] = float("-inf")
+    x[5, 200] = float("nan")
+    x[4, 0:8] = torch.tensor([-0.0, 0.0, -0.0, 0.0, 1e18, -1e18, 1.0, 1.0])
+    X = x.to(torch.bfloat16)
+    vq, meta, rs = lx.prune_compress_fp8(X.cuda(), 1)
+    ov, om, oact = oracle.compress_fp8(u16(X))
+    got = vq.cpu().numpy()
+    gd, od = oracle.e4m3_decode(got), oracle.e4m3_decode(ov)
+    nan = np.isnan(od)
+    assert (np.isnan(gd) == nan).all()
+    assert (got[~nan] == ov[~nan]).all()
+    assert (meta.cpu().numpy() == oracle.meta_canon_to_hw_fp8(om, M, K)).all()
+    ref = oracle.row_scale(u16(X), 1).astype(np.float64) * oact.astype(np.float64)
+    got_s = rs.cpu().numpy().astype(np.float64)
+    fin = np.isfinite(ref)
+    assert (np.isfinite(got_s) == fin).all()
+    np.testing.assert_allclose(got_s[fin], ref[fin], rtol=1e-5)
+
+
+@pytest.mark.parametrize("ring", ["0", "1", "2", "4", "8"])
+def test_every_fp8_prune_form_gives_the_same_codes(ring, monkeypatch):
+    """The 16-rows-per-CTA kernel and every warp split of the single-read kernel."""
+    from paper_2605_26632_b200 import binding
+
+    monkeypatch.setenv("LYNX_FP8_RING", ring)
+    ctx = binding.Lynx(0)
+    try:
+        M, K = 333, 4096
+        X = inputs.make_x(M, K, "outlier", 777)
+        ov, om, oact = oracle.compress_fp8(u16(X))
+        vq, meta, rs = ctx.prune_compress_fp8(X.cuda(), 1)
+        assert (vq.cpu().numpy() == ov).all()
+        assert (meta.cpu().numpy() == oracle.meta_canon_to_hw_fp8(om, M, K)).all()
+        ref = oracle.row_scale(u16(X), 1).astype(np.float64) * oact.astype(np.float64)
+        np.testing.assert_allclose(rs.cpu().numpy(), ref, rtol=1e-5)
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
+
+
 @pytest.mark.parametrize("M,K,mode", [(300, 1024, 1), (129, 256, 0), (2048, 3072, 1)])
 def test_supplied_row_maximum(lx, M, K, mode):
     """The true maxima supplied by the caller give the same bits as the two-pass form; a
