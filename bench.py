@@ -52,6 +52,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-lora", action="store_true", help="skip the extra measurement of the layer with the low-rank branch")
+    ap.add_argument("--no-fp8", action="store_true", help="skip the extra measurement of the layer on FP8 operands")
     return ap.parse_args()
 
 
@@ -380,6 +381,30 @@ def main():
                 "how": "lynx_act_sparse_linear_lora: prune/compress + sparse GEMM whose launch also computes "
                        "T = (X L_B^T) / s and adds T L_A^T in its accumulator"}
 
+    # the same layer on FP8 (E4M3) operands, outside the headline number: weights quantised once
+    # (symmetric per output channel), activations pruned and quantised (per-row scale found in the
+    # data) inside every step; same rotation and event timing
+    fp8 = None
+    if not args.no_fp8 and comp_mode in (0, 1):
+        Wqs = [lx.quantize_weights_fp8(w, True) for w in Ws]
+        for i in range(3):
+            lx.act_sparse_linear_fp8(Xs[i % NSETS], Wqs[i % NSETS][0], Wqs[i % NSETS][1], bias, comp_mode, None,
+                                     Ys[i % NSETS])
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for i in range(args.steps):
+            j = i % NSETS
+            lx.act_sparse_linear_fp8(Xs[j], Wqs[j][0], Wqs[j][1], bias, comp_mode, None, Ys[j])
+        f1.record(stream)
+        torch.cuda.synchronize()
+        fp8_ms = f0.elapsed_time(f1) / args.steps
+        fp8 = {"ms_per_step": fp8_ms, "tflops_dense_equivalent": 2.0 * M * N * K / (fp8_ms * 1e-3) / 1e12,
+               "speedup_vs_step": (total_ms / args.steps) / fp8_ms, "speedup_vs_dense_bf16": dense_ms / fp8_ms,
+               "dtype": "e4m3 operands, f32 accumulation, bf16 output",
+               "how": "lynx_act_sparse_linear_fp8: single-read quantising prune/compress + kind::f8f6f4 sparse GEMM"}
+        del Wqs
+
     # end to end through the host-buffer entry point: pinned X in, pinned Y out, every step
     e2e = None
     if not args.no_e2e:
@@ -455,6 +480,7 @@ def main():
         "clocks": clocks,
         "e2e": e2e,
         "lora": lora,
+        "fp8": fp8,
         "gpu_launches": int(launches),
     }
 
