@@ -434,6 +434,53 @@ def test_other_dit_family_shapes(lx, K, N):
     _full_size_case(lx, inputs.sweep_workload(inputs.OTHER_FAMILY_M, K, N, idx), 16)
 
 
+def test_more_than_2_to_the_31_elements(lx):
+    """M x K = 176128 x 12288 > 2^31 elements (X alone is 4.3 GB): every offset in the prune kernels,
+    the tensor maps and the GEMM has to be 64-bit.  The rows are 43 copies of one 4096-row matrix
+    scaled by powers of two; the oracle sees the sampled rows as they sit on the device."""
+    K, N, base_rows, copies = 12288, 256, 4096, 43
+    M = base_rows * copies
+    assert M * K > 2 ** 31 and M % 128 == 0
+    base = inputs.make_x(base_rows, K, "outlier", 4242).cuda()
+    X = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    for c in range(copies):
+        X[c * base_rows:(c + 1) * base_rows] = base * (2.0 ** ((c % 7) - 3))
+    W, b = inputs.make_w(N, K, 4243), inputs.make_bias(N, 4243)
+    edge = (2 ** 31) // K                     # the row in which element offset 2^31 falls
+    rows = np.unique(np.concatenate([[0, 1, edge - 1, edge, edge + 1, M - 2, M - 1],
+                                     np.random.default_rng(7).choice(M, 25, replace=False)])).astype(np.int64)
+    ridx = torch.from_numpy(rows).cuda()
+    Xs = u16(X[ridx].cpu())
+    ov, om = oracle.compress(Xs)
+    values, meta, scale = lx.prune_compress(X, 1)
+    assert (u16(values[ridx].cpu()) == ov).all()
+    canon = lx.meta_to_canonical(meta, M, K)
+    assert (canon[ridx].cpu().numpy().view(np.uint16) == om.view(np.uint16)).all()
+    np.testing.assert_allclose(scale[ridx].cpu().numpy(), oracle.row_scale(Xs, 1), rtol=SCALE_RTOL)
+    Y = lx.sparse_linear(values, meta, W.cuda(), b.cuda(), scale)
+    ref = oracle.act_sparse_linear(Xs, u16(W), bias=u16(b), comp_mode=1)
+    check_y(Y[ridx], ref["Y"])
+    Y2 = lx.act_sparse_linear(X, W.cuda(), b.cuda(), 1)
+    assert torch.equal(Y, Y2)
+    del values, meta, canon, Y2
+    # the FP8 quantising prune on the same rows (single-read kernel, two warps per row)
+    vq, meta8, rs8 = lx.prune_compress_fp8(X, 1)
+    oq, om8, oact = oracle.compress_fp8(Xs)
+    assert (vq[ridx].cpu().numpy() == oq).all()
+    hw = oracle.meta_canon_to_hw_fp8(om8, len(rows), K)          # rows 0.. of one 128-row block
+    kb = torch.arange(K // 128, device="cuda").view(1, -1, 1)
+    byte = torch.arange(16, device="cuda").view(1, 1, -1)
+    r = ridx.view(-1, 1, 1)
+    got = meta8[((r // 128) * (K // 128) + kb) * 2048 + (r % 128) * 16 + byte].cpu().numpy()
+    i = np.arange(len(rows)).reshape(-1, 1, 1)
+    want = hw[(kb.cpu().numpy()) * 2048 + i * 16 + byte.cpu().numpy()]
+    assert (got == want).all()
+    ref8 = oracle.row_scale(Xs, 1).astype(np.float64) * oact.astype(np.float64)
+    np.testing.assert_allclose(rs8[ridx].cpu().numpy(), ref8, rtol=1e-5)
+    torch.cuda.synchronize()
+    assert lx.last_error() == 0
+
+
 # ------------------------------------------------------------------ host-side error reporting ---
 
 def test_argument_errors_are_reported_not_launched(lx):
