@@ -182,13 +182,13 @@ lora_down_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             // hand-over: every drain thread's partial rows are written, then one ticket per CTA
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (warp == 2 && lane == 0) {
-                __threadfence();
-                const uint32_t t = atomicAdd(p.tickets + tm, 1u);
+                // one acquire-release add: publishes this CTA's partial rows (ordered before it by
+                // the barrier) and, for the CTA that draws the last ticket, makes all others' visible
+                const uint32_t t = atom_add_acq_rel_gpu(p.tickets + tm, 1u);
                 if (t == (uint32_t)p.splits - 1) {
                     p.tickets[tm] = 0;  // ready for the next launch
                     *s_last = 1;
                 }
-                __threadfence();
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
             // a CTA that timed out still takes its ticket (so nobody is left waiting); the error

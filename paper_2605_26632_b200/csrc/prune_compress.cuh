@@ -317,18 +317,18 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
             *reinterpret_cast<float2*>(mine + 2 * (r + 8)) = make_float2(numB, denB);
         }
         // The last CTA of the row block to get here adds all partial sums, in a fixed order.  One
-        // thread fences and takes the ticket for the whole CTA (the barrier makes the other
-        // warps' stores its predecessors), so only its warp waits for the stores to drain.
+        // thread takes the ticket for the whole CTA (the barrier makes the other warps' stores
+        // its predecessors), so only its warp waits for the stores to drain.
         __syncthreads();
         if (tid == 0) {
-            __threadfence();
-            const uint32_t t = atomicAdd(&tickets[rb16], 1u);
+            // release: this CTA's partial sums (ordered before by the barrier) are visible to whoever
+            // reads a later ticket value; acquire: the last CTA sees every earlier CTA's sums
+            const uint32_t t = atom_add_acq_rel_gpu(&tickets[rb16], 1u);
             s_last = (t == (uint32_t)(ctas_per_rb - 1)) ? 1u : 0u;
         }
         __syncthreads();
         if (active) prune_tile_store(last, va, vb, slab, okA, okB);
         if (!s_last) return;
-        __threadfence();
         const int row = tid & 15, jl = tid >> 4;  // 16 rows x (PRUNE_CTA_WARPS * 2) strided sums
         const float2* pp = reinterpret_cast<const float2*>(partial) + rb16 * KS * 16 + row;
         float num = 0.f, den = 0.f;
