@@ -227,19 +227,27 @@ LYNX_API lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_ho
  *   low-rank workspace (fp32 partials of the K splits; grown on demand, see lynx_reserve_lora)
  *   and a ticket word per 128-row block (M <= 2097152).  The result does not depend on the
  *   order in which CTAs finish.
+ * lynx_prune_compress_lora:  lynx_prune_compress and lynx_lora_down in ONE launch that reads X
+ *   once: values and meta as lynx_prune_compress writes them (bit for bit), T as above with s_m
+ *   the per-row norm compensation (mode LYNX_COMP_ROW) or 1 (LYNX_COMP_NONE; other modes:
+ *   LYNX_ERR_INVALID_ARG).  Under LYNX_COMP_ROW the row sums stay on the context, exactly as
+ *   after lynx_prune_compress with LYNX_ROW_SCALE_DEFERRED: pass comp->row_scale =
+ *   LYNX_ROW_SCALE_DEFERRED to the lynx_sparse_linear_lora call that follows.
  * lynx_sparse_linear_lora:  lynx_sparse_linear plus the T L_A^T term; T must come from
- *   lynx_lora_down called with the same row_scale that comp carries.
- * lynx_act_sparse_linear_lora:  the whole layer, intermediates in the context's scratch.  For
- *   R = 64 it is two launches: prune/compress, then a sparse GEMM launch that first computes T
- *   itself (its clusters share the (row block, K split) items of X L_B^T, publish the T rows
- *   through ready words, and wait -- bounded -- for the rows a tile needs) and then runs the
- *   tiles with the low-rank steps.  Otherwise (R = 128) three launches: prune/compress,
- *   lynx_lora_down, lynx_sparse_linear_lora.  Both give Y within the stated tolerance of the
- *   definition; they may differ from each other in the last bit of T (different K splits, and
- *   the in-launch form multiplies by 1/s_m where lynx_lora_down divides).
+ *   lynx_lora_down called with the same row_scale that comp carries, or from
+ *   lynx_prune_compress_lora (deferred row scale).
+ * lynx_act_sparse_linear_lora:  the whole layer, intermediates in the context's scratch: two
+ *   launches, lynx_prune_compress_lora's kernel and the sparse GEMM with the low-rank steps
+ *   (LYNX_COMP_NONE / LYNX_COMP_ROW; the other modes take prune/compress, lynx_lora_down and the
+ *   GEMM as three launches).  Y is within the stated tolerance of the definition whichever form
+ *   computed T (they may differ in the last bit of T: different K splits).
  * Pointers and leading dimensions follow the 16-byte rule of the other entry points.
  */
 LYNX_API lynx_status lynx_reserve_lora(lynx_ctx* ctx, int64_t M, int64_t K, int64_t R);
+LYNX_API lynx_status lynx_prune_compress_lora(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
+                                              int64_t ldx, const void* LB, int64_t R, int64_t ldlb,
+                                              void* values, void* meta, lynx_comp_mode mode, void* T,
+                                              int64_t ldt, void* stream);
 LYNX_API lynx_status lynx_lora_down(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx,
                                     const void* LB, int64_t R, int64_t ldlb, const float* row_scale,
                                     void* T, int64_t ldt, void* stream);

@@ -22,7 +22,7 @@ EXPORTS = [
     "lynx_meta_bytes", "lynx_workspace_bytes", "lynx_reserve", "lynx_prune_compress",
     "lynx_sparse_linear", "lynx_act_sparse_linear", "lynx_act_sparse_linear_host",
     "lynx_meta_to_canonical", "lynx_decompress", "lynx_launch_count", "lynx_prune_compress_static",
-    "lynx_reserve_lora", "lynx_lora_down", "lynx_sparse_linear_lora", "lynx_act_sparse_linear_lora",
+    "lynx_reserve_lora", "lynx_lora_down", "lynx_prune_compress_lora", "lynx_sparse_linear_lora", "lynx_act_sparse_linear_lora",
     "lynx_quantize_weights_fp8", "lynx_prune_compress_fp8", "lynx_sparse_linear_fp8",
     "lynx_act_sparse_linear_fp8",
 ]
@@ -89,6 +89,7 @@ def load_library() -> ctypes.CDLL:
     lib.lynx_prune_compress_static.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
     lib.lynx_reserve_lora.argtypes = [vp, i64, i64, i64]
     lib.lynx_lora_down.argtypes = [vp, vp, i64, i64, i64, vp, i64, i64, vp, vp, i64, vp]
+    lib.lynx_prune_compress_lora.argtypes = [vp, vp, i64, i64, i64, vp, i64, i64, vp, vp, ctypes.c_int, vp, i64, vp]
     lib.lynx_sparse_linear_lora.argtypes = [vp, vp, vp, i64, i64, vp, i64, i64, vp, ctypes.POINTER(_Comp), vp,
                                             i64, vp, i64, i64, vp, i64, vp]
     lib.lynx_act_sparse_linear_lora.argtypes = [vp, vp, i64, i64, i64, vp, i64, i64, vp, vp, i64, vp, i64, i64,
@@ -268,6 +269,25 @@ class Lynx:
                                         _ptr(row_scale), _ptr(out), out.stride(0), _stream()), "lynx_lora_down")
         return out
 
+    def prune_compress_lora(self, X: torch.Tensor, LB: torch.Tensor, mode: int = COMP_NONE, values=None, meta=None,
+                            T=None):
+        """One launch, X read once -> (values, meta, T = (X L_B^T) / s); under COMP_ROW the row sums stay
+        on the context: pass ROW_SCALE_DEFERRED to the sparse_linear_lora call that follows."""
+        _bf16_2d(X, "X")
+        _bf16_2d(LB, "LB")
+        M, K = X.shape
+        R = LB.shape[0]
+        if values is None:
+            values = torch.empty((M, K // 2), dtype=torch.bfloat16, device=X.device)
+        if meta is None:
+            meta = torch.empty(meta_bytes(M, K), dtype=torch.uint8, device=X.device)
+        if T is None:
+            T = torch.empty((M, R), dtype=torch.bfloat16, device=X.device)
+        _check(self._lib.lynx_prune_compress_lora(self._h, _ptr(X), M, K, X.stride(0), _ptr(LB), R, LB.stride(0),
+                                                  _ptr(values), _ptr(meta), mode, _ptr(T), T.stride(0), _stream()),
+               "lynx_prune_compress_lora")
+        return values, meta, T
+
     def sparse_linear_lora(self, values: torch.Tensor, meta: torch.Tensor, W: torch.Tensor, T: torch.Tensor,
                            LA: torch.Tensor, bias=None, row_scale=None, residual=None, out=None) -> torch.Tensor:
         _bf16_2d(values, "values")
@@ -279,7 +299,7 @@ class Lynx:
         R = LA.shape[1]
         if out is None:
             out = torch.empty((M, N), dtype=torch.bfloat16, device=values.device)
-        comp = _Comp(None if row_scale is None else row_scale.data_ptr(),
+        comp = _Comp(1 if row_scale is ROW_SCALE_DEFERRED else (None if row_scale is None else row_scale.data_ptr()),
                      None if residual is None else residual.data_ptr(),
                      0 if residual is None else residual.stride(0))
         _check(self._lib.lynx_sparse_linear_lora(self._h, _ptr(values), _ptr(meta), M, K, _ptr(W), N, W.stride(0),

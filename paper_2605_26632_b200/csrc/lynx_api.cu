@@ -15,6 +15,7 @@
 #include "fused_linear.cuh"
 #include "lora_down.cuh"
 #include "fp8_path.cuh"
+#include "prune_lora.cuh"
 
 using namespace lynx;
 
@@ -39,7 +40,7 @@ struct lynx_ctx {
     uint32_t l0_done_total = 0;   // groups published by all such launches so far (mod 2^32)
     int l0_force_splits = 0, l0_force_fill = -1;  // development overrides of the phase-0 plan
     int defer_scale = 1;  // layer calls: row scale summed in the GEMM epilogue (LYNX_DEFER_SCALE=0: in the prune kernel)
-    int lora_fuse = 1;            // down projection inside the GEMM launch when the tile allows (LYNX_LORA_FUSE=0: own kernel)
+    int lora_fuse = 2;            // down projection: 2 = in the prune launch (X read once), 1 = inside the GEMM launch, 0 = own kernel
     float* sk_partial = nullptr;  // stream-K partial tiles (one slot per cluster) + ready words
     uint32_t* sk_flags = nullptr;
     uint32_t sk_epoch = 0;
@@ -50,6 +51,7 @@ struct lynx_ctx {
     int prune_tpu = 0;  // 0 = auto
     int fp8_ring = 1;   // FP8 activations: single-read ring kernel (LYNX_FP8_RING=0: one CTA per 16 rows)
     int fp8_ring_forced = 0;
+    int pl_force_splits = 0;  // development override: cluster size of the prune + down-projection kernel
     std::mutex mu;
 };
 
@@ -606,6 +608,101 @@ lynx_status launch_lora_down(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
     return LYNX_OK;
 }
 
+// K splits of the prune + down-projection kernel (128-element K blocks) = CTAs per cluster, 1..8.
+// Every CTA holds a whole SM; `cap[i]` = CTAs of clusters of i + 1 that the GPU holds at once.
+void prune_lora_plan(const int cap[8], int64_t M, int64_t K, int* splits, int* kb_per_split) {
+    const int tiles_m = (int)((M + 127) / 128), kblocks = (int)(K / 128);
+    int best_s = 1, best_per = kblocks;
+    double best = 1e30;
+    for (int i = 0; i < 8; ++i) {
+        const int sp = i + 1;
+        if (sp > kblocks) break;
+        if (cap[i] < sp) continue;
+        const int per = (kblocks + sp - 1) / sp;
+        if ((kblocks + per - 1) / per != sp) continue;  // every CTA of the cluster needs a K block
+        const double rounds = (double)(((int64_t)tiles_m * sp + cap[i] - 1) / cap[i]);
+        const double t = rounds * (per + 4.0);
+        if (t < best) { best = t; best_s = sp; best_per = per; }
+    }
+    *splits = best_s;
+    *kb_per_split = best_per;
+}
+
+template <class Cfg, bool SUMS>
+lynx_status launch_prune_lora(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, const void* LB,
+                              int64_t ldlb, void* values, void* meta, float* scale_partial, void* T, int64_t ldt,
+                              cudaStream_t st, int* splits_out) {
+    CUtensorMap tx, tlb;
+    if (!make_tmap_2d(&tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx * 2, 64,
+                      Cfg::BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tlb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, LB, (uint64_t)Cfg::R, (uint64_t)K,
+                      (uint64_t)ldlb * 2, 64, Cfg::R, CU_TENSOR_MAP_SWIZZLE_128B))
+        return LYNX_ERR_CUDA;
+    auto kern = prune_lora_kernel<Cfg, SUMS>;
+    static bool attr_set[MAX_CTX_DEVICES] = {};  // per instantiation
+    if (lynx_status as = allow_dynamic_smem(kern, Cfg::SMEM_BYTES, ctx->device, attr_set); as != LYNX_OK) return as;
+    // how many CTAs of clusters of 1..8 fit on the GPU at once (asked once per device)
+    static int caps[MAX_CTX_DEVICES][8] = {};
+    int* cap = caps[ctx->device];
+    if (cap[0] == 0) {
+        for (int i = 0; i < 8; ++i) {
+            cudaLaunchConfig_t qc = {};
+            qc.gridDim = dim3((unsigned)(ctx->num_sms / (i + 1) * (i + 1)));
+            qc.blockDim = dim3(Cfg::THREADS);
+            qc.dynamicSmemBytes = Cfg::SMEM_BYTES;
+            cudaLaunchAttribute qa[1];
+            qa[0].id = cudaLaunchAttributeClusterDimension;
+            qa[0].val.clusterDim.x = (unsigned)(i + 1);
+            qa[0].val.clusterDim.y = 1;
+            qa[0].val.clusterDim.z = 1;
+            qc.attrs = qa;
+            qc.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kern, &qc) != cudaSuccess) n = 0;
+            cap[i] = n * (i + 1);
+        }
+        if (cap[0] <= 0) cap[0] = ctx->num_sms;
+        if (getenv("LYNX_DEBUG_PLAN"))
+            fprintf(stderr, "prune+down: CTAs resident by cluster size 1..8: %d %d %d %d %d %d %d %d\n", cap[0], cap[1],
+                    cap[2], cap[3], cap[4], cap[5], cap[6], cap[7]);
+    }
+    PruneLoraParams p;
+    p.M = M; p.K = K;
+    prune_lora_plan(cap, M, K, &p.splits, &p.kb_per_split);
+    if (const int f = ctx->pl_force_splits; f >= 1 && f <= 8 && cap[f - 1] >= f) {
+        const int kblocks = (int)(K / 128), per = (kblocks + f - 1) / f;
+        if (f <= kblocks && (kblocks + per - 1) / per == f) {  // every CTA of the cluster gets a K block
+            p.splits = f;
+            p.kb_per_split = per;
+        }
+    }
+    p.values = static_cast<uint16_t*>(values);
+    p.meta = static_cast<uint8_t*>(meta);
+    p.scale_partial = scale_partial;
+    p.T = static_cast<uint16_t*>(T);
+    p.ldt = ldt;
+    p.dev_error = ctx->err_dev;
+    const int tiles_m = (int)((M + Cfg::BM - 1) / Cfg::BM);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(tiles_m * p.splits));
+    cfg.blockDim = dim3(Cfg::THREADS);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)p.splits;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, kern, tx, tlb, p) != cudaSuccess) return LYNX_ERR_CUDA;
+    ctx->launches++;
+    *splits_out = p.splits;
+    return LYNX_OK;
+}
+
 lynx_status check_lora_rank(int64_t R) {
     if (R < 1) return LYNX_ERR_INVALID_ARG;
     if (R != 64 && R != 128) return LYNX_ERR_UNSUPPORTED_SHAPE;
@@ -650,7 +747,7 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
     if (env) ctx->pdl = atoi(env);
     env = getenv("LYNX_STREAMK");  // 1 turns the stream-K tail on
     if (env) ctx->streamk = atoi(env);
-    env = getenv("LYNX_LORA_FUSE");  // 0: down projection of the low-rank branch as its own kernel
+    env = getenv("LYNX_LORA_FUSE");  // down projection of the low-rank branch: 0 own kernel, 1 in the GEMM launch, 2 in the prune launch
     if (env) ctx->lora_fuse = atoi(env);
     env = getenv("LYNX_L0_SPLITS");  // development overrides: K splits of the in-GEMM down projection,
     if (env) ctx->l0_force_splits = atoi(env);
@@ -660,6 +757,8 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
     if (env) ctx->defer_scale = atoi(env);
     env = getenv("LYNX_PRUNE_TPU");  // development override: 128-element K blocks per warp
     if (env) ctx->prune_tpu = atoi(env);
+    env = getenv("LYNX_PL_SPLITS");  // development override: K splits (= cluster size) of the prune + down-projection kernel
+    if (env) ctx->pl_force_splits = atoi(env);
     env = getenv("LYNX_FP8_RING");  // development override: 0 = one CTA per 16 rows, n = ring with n warps per row
     if (env) {
         ctx->fp8_ring = atoi(env);
@@ -1007,6 +1106,55 @@ lynx_status lynx_lora_down(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, i
     return launch_lora_down<LoraDownCfg<128>>(ctx, X, M, K, ldx, LB, ldlb, row_scale, T, ldt, partial, st);
 }
 
+// Prune / compress + row sums + T = (X L_B^T) / s in one launch (X read once).  The row sums stay
+// in the context's scratch for the GEMM that follows (deferred row scale); *ss names them.
+static lynx_status prune_lora_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, const void* LB,
+                                   int64_t R, int64_t ldlb, void* values, void* meta, lynx_comp_mode mode, void* T,
+                                   int64_t ldt, void* stream, ScaleSrc* ss) {
+    lynx_status s = check_common(ctx, M, K);
+    if (s != LYNX_OK) return s;
+    if ((s = check_lora_rank(R)) != LYNX_OK) return s;
+    if (!X || !LB || !values || !meta || !T) return LYNX_ERR_INVALID_ARG;
+    if (mode != LYNX_COMP_NONE && mode != LYNX_COMP_ROW) return LYNX_ERR_INVALID_ARG;
+    if (ldx < K || ldlb < K || ldt < R) return LYNX_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(LB) || !aligned16(T) || !aligned16(meta) || (ldx % 8) || (ldlb % 8) || (ldt % 8) ||
+        (reinterpret_cast<uintptr_t>(values) & 31u))
+        return LYNX_ERR_ALIGNMENT;
+    const ScratchLayout L = scratch_layout(M, 8, K);
+    {
+        std::lock_guard<std::mutex> lock(ctx->mu);
+        if (ctx->scratch_bytes < L.prune_end && (s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
+    }
+    if ((s = check_device_error(ctx)) != LYNX_OK) return s;
+    float* spart = reinterpret_cast<float*>(static_cast<char*>(ctx->scratch) + L.partial);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int splits = 0;
+    const bool sums = mode == LYNX_COMP_ROW;
+    if (R == 64)
+        s = sums ? launch_prune_lora<PruneLoraCfg<64>, true>(ctx, X, M, K, ldx, LB, ldlb, values, meta, spart, T, ldt, st, &splits)
+                 : launch_prune_lora<PruneLoraCfg<64>, false>(ctx, X, M, K, ldx, LB, ldlb, values, meta, nullptr, T, ldt, st, &splits);
+    else
+        s = sums ? launch_prune_lora<PruneLoraCfg<128>, true>(ctx, X, M, K, ldx, LB, ldlb, values, meta, spart, T, ldt, st, &splits)
+                 : launch_prune_lora<PruneLoraCfg<128>, false>(ctx, X, M, K, ldx, LB, ldlb, values, meta, nullptr, T, ldt, st, &splits);
+    if (s != LYNX_OK) return s;
+    // the scratch's sums now belong to this call, in this kernel's split count
+    ctx->deferred_partial = sums ? spart : nullptr;
+    ctx->deferred_ks = sums ? splits : 0;
+    ctx->deferred_M = M;
+    ctx->deferred_K = K;
+    if (ss) {
+        ss->partial = ctx->deferred_partial;
+        ss->ks = ctx->deferred_ks;
+    }
+    return LYNX_OK;
+}
+
+lynx_status lynx_prune_compress_lora(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx, const void* LB,
+                                     int64_t R, int64_t ldlb, void* values, void* meta, lynx_comp_mode mode, void* T,
+                                     int64_t ldt, void* stream) {
+    return prune_lora_impl(ctx, X, M, K, ldx, LB, R, ldlb, values, meta, mode, T, ldt, stream, nullptr);
+}
+
 lynx_status lynx_sparse_linear_lora(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
                                     const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
                                     const void* T, int64_t ldt, const void* LA, int64_t R, int64_t ldla, void* Y,
@@ -1015,7 +1163,6 @@ lynx_status lynx_sparse_linear_lora(lynx_ctx* ctx, const void* values, const voi
     if (s != LYNX_OK) return s;
     if ((s = check_lora_rank(R)) != LYNX_OK) return s;
     if (!values || !meta || !W || !Y || !T || !LA || N < 8) return LYNX_ERR_INVALID_ARG;
-    if (comp && comp->row_scale == LYNX_ROW_SCALE_DEFERRED) return LYNX_ERR_INVALID_ARG;  // T needs the finished scale
     if (N % 8 != 0) return LYNX_ERR_UNSUPPORTED_SHAPE;
     if (ldw < K || ldy < N || ldt < R || ldla < R) return LYNX_ERR_INVALID_ARG;
     if (!aligned16(values) || !aligned16(meta) || !aligned16(W) || !aligned16(Y) || !aligned16(T) || !aligned16(LA) ||
@@ -1028,6 +1175,17 @@ lynx_status lynx_sparse_linear_lora(lynx_ctx* ctx, const void* values, const voi
     }
     if ((s = check_device_error(ctx)) != LYNX_OK) return s;
     LoraArgs lora{T, ldt, LA, ldla, (int)R};
+    if (comp && comp->row_scale == LYNX_ROW_SCALE_DEFERRED) {
+        // the sums lynx_prune_compress_lora left on the context (T was divided by the same scale)
+        if (!ctx->deferred_partial || ctx->deferred_M != M || ctx->deferred_K != K) return LYNX_ERR_INVALID_ARG;
+        ScaleSrc ss;
+        ss.partial = ctx->deferred_partial;
+        ss.ks = ctx->deferred_ks;
+        lynx_comp c2 = *comp;
+        c2.row_scale = nullptr;
+        return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &c2, &lora, Y, ldy,
+                           static_cast<cudaStream_t>(stream), 0, &ss);
+    }
     return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, comp, &lora, Y, ldy,
                        static_cast<cudaStream_t>(stream));
 }
@@ -1061,6 +1219,20 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
     float* scale = sums_needed(mode) ? reinterpret_cast<float*>(base + L.scale) : nullptr;
     void* T = static_cast<char*>(ctx->lora_ws) + LL.T;
     const int cfg = pick_gemm_cfg(ctx, M, N, K, (int)(R / 64));
+    if (ctx->lora_fuse == 2 && (mode == LYNX_COMP_NONE || (mode == LYNX_COMP_ROW && ctx->defer_scale != 0))) {
+        // two launches, X read once: prune / compress + row sums + T in the first, the GEMM (which
+        // finishes the row scale in its epilogue and adds T L_A^T in its accumulator) in the second
+        ScaleSrc ss2;
+        if ((s = prune_lora_impl(ctx, X, M, K, ldx, LB, R, ldlb, values, meta, mode, T, R, stream, &ss2)) != LYNX_OK)
+            return s;
+        lynx_comp comp2;
+        comp2.row_scale = nullptr;
+        comp2.residual = residual;
+        comp2.ldr = ldr;
+        LoraArgs lora2{T, R, LA, ldla, (int)R};
+        return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &comp2, &lora2, Y, ldy,
+                           static_cast<cudaStream_t>(stream), cfg, &ss2);
+    }
     const bool groups_fit = (size_t)((M + 255) / 256) * 8 * 4 <= L0_WORDS_BYTES;
     const bool fused = ctx->lora_fuse && R == 64 && cfg_supports_l0(cfg) && !ctx->streamk && groups_fit;
     // (the separate down-projection kernel reads row_scale, so the scale is only deferred when the

@@ -169,28 +169,14 @@ struct TileOut {
     uint32_t w0, w1;        // the lane's two metadata words
 };
 
-template <bool SUMS, bool GUARD, bool GROUP = false>
-__device__ __forceinline__ void prune_tile_compute(const uint16_t* xa, const uint16_t* xb, bool okA, bool okB,
-                                                   const uint32_t* lut, TileOut& out, float& numA, float& denA,
-                                                   float& numB, float& denB) {
-    uint32_t a0[8], a1[8], b0[8], b1[8];
-    if constexpr (GUARD) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) a0[i] = a1[i] = b0[i] = b1[i] = 0u;
-        if (okA) {
-            ldg256_stream(xa, a0);
-            ldg256_stream(xa + 16, a1);
-        }
-        if (okB) {
-            ldg256_stream(xb, b0);
-            ldg256_stream(xb + 16, b1);
-        }
-    } else {
-        ldg256_stream(xa, a0);
-        ldg256_stream(xa + 16, a1);
-        ldg256_stream(xb, b0);
-        ldg256_stream(xb + 16, b1);
-    }
+// Selection, compression and (SUMS) the row sums of one 16 x 128 tile whose elements are already in
+// registers: a0 / a1 = elements 0..15 / 16..31 of this lane's 32-element slice of row r, b0 / b1 the
+// same of row r + 8.
+template <bool SUMS, bool GROUP = false>
+__device__ __forceinline__ void prune_tile_core(const uint32_t (&a0)[8], const uint32_t (&a1)[8],
+                                                const uint32_t (&b0)[8], const uint32_t (&b1)[8],
+                                                const uint32_t* lut, TileOut& out, float& numA, float& denA,
+                                                float& numB, float& denB) {
     const uint32_t ma0 = prune_vec16(a0, lut, out.oa);
     const uint32_t ma1 = prune_vec16(a1, lut, out.oa + 4);
     const uint32_t mb0 = prune_vec16(b0, lut, out.ob);
@@ -221,6 +207,31 @@ __device__ __forceinline__ void prune_tile_compute(const uint16_t* xa, const uin
             denB = fma_sq_bf16x2(out.ob[i], denB);
         }
     }
+}
+
+template <bool SUMS, bool GUARD, bool GROUP = false>
+__device__ __forceinline__ void prune_tile_compute(const uint16_t* xa, const uint16_t* xb, bool okA, bool okB,
+                                                   const uint32_t* lut, TileOut& out, float& numA, float& denA,
+                                                   float& numB, float& denB) {
+    uint32_t a0[8], a1[8], b0[8], b1[8];
+    if constexpr (GUARD) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a0[i] = a1[i] = b0[i] = b1[i] = 0u;
+        if (okA) {
+            ldg256_stream(xa, a0);
+            ldg256_stream(xa + 16, a1);
+        }
+        if (okB) {
+            ldg256_stream(xb, b0);
+            ldg256_stream(xb + 16, b1);
+        }
+    } else {
+        ldg256_stream(xa, a0);
+        ldg256_stream(xa + 16, a1);
+        ldg256_stream(xb, b0);
+        ldg256_stream(xb + 16, b1);
+    }
+    prune_tile_core<SUMS, GROUP>(a0, a1, b0, b1, lut, out, numA, denA, numB, denB);
 }
 
 __device__ __forceinline__ void prune_tile_store(const TileOut& out, uint16_t* va, uint16_t* vb, uint32_t* slab,

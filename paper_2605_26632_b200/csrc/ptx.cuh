@@ -232,6 +232,15 @@ __device__ __forceinline__ uint32_t mapa(uint32_t smem_addr, uint32_t rank) {
     return r;
 }
 
+// 16-byte load from the shared memory of any CTA of the cluster (address from mapa)
+__device__ __forceinline__ float4 lds128_cluster_f32(uint32_t cluster_addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(cluster_addr));
+    return v;
+}
+
 // ---------------------------------------------------------------------------- tcgen05 --------
 
 template <int CG>

@@ -84,6 +84,97 @@ def test_lora_down_matches_oracle(lx, M, K, R, mode):
     assert torch.equal(T, T2)
 
 
+@pytest.mark.parametrize("M,K,R,mode", [
+    (256, 512, 64, 0), (256, 512, 64, 1), (300, 1024, 64, 1), (129, 128, 64, 1), (1, 128, 64, 1),
+    (1000, 3072, 128, 1), (700, 1664, 128, 0), (4096, 3072, 64, 1), (2048, 12288, 64, 1), (4352, 3072, 64, 0),
+])
+def test_prune_compress_lora_one_pass(lx, M, K, R, mode):
+    """Prune / compress and the down projection in one launch (X read once): values and metadata
+    bit for bit, T within a bf16 rounding, the row sums good for the GEMM that follows."""
+    from paper_2605_26632_b200 import binding
+
+    X = inputs.make_x(M, K, "outlier", 60 + M)
+    N = 264
+    W, b = inputs.make_w(N, K, 61 + M), inputs.make_bias(N, 61 + M)
+    LA, LB = inputs.make_lora(N, K, R, 62 + M)
+    Xc = X.cuda()
+    values, meta, T = lx.prune_compress_lora(Xc, LB.cuda(), mode)
+    ov, om = oracle.compress(u16(X))
+    assert (u16(values) == ov).all(), "values differ"
+    assert (meta.cpu().numpy() == oracle.meta_canon_to_hw(om, M, K)).all(), "metadata differs"
+    ref = oracle_t(X, LB, mode)
+    got = T.float().cpu().numpy()
+    tol = 2.0 ** -8 * np.abs(ref) + 1e-5 * np.abs(ref).max()
+    assert (np.abs(got - ref) <= tol).all(), float(np.abs(got - ref).max())
+    # the GEMM that follows takes the row sums the launch left on the context
+    Y = lx.sparse_linear_lora(values, meta, W.cuda(), T, LA.cuda(), b.cuda(),
+                              binding.ROW_SCALE_DEFERRED if mode else None)
+    yref = oracle.act_sparse_linear_lora(u16(X), u16(W), u16(LA), u16(LB), bias=u16(b), comp_mode=mode)
+    check_y(Y, yref["Y"])
+    # reproducible whichever CTA finishes a row block, and the layer call is these two launches
+    values2, meta2, T2 = lx.prune_compress_lora(Xc, LB.cuda(), mode)
+    assert torch.equal(T, T2) and torch.equal(values, values2) and torch.equal(meta, meta2)
+    Y2 = lx.act_sparse_linear_lora(Xc, W.cuda(), LA.cuda(), LB.cuda(), b.cuda(), mode)
+    assert torch.equal(Y, Y2)
+
+
+@pytest.mark.parametrize("splits,K", [(1, 3584), (2, 3584), (3, 3584), (4, 3584), (5, 3584), (6, 3584), (7, 3584),
+                                      (8, 4096)])
+def test_prune_compress_lora_every_cluster_size(splits, K, monkeypatch):
+    """The K splits of a row block form a cluster of 1..8 CTAs that add their partials through
+    distributed shared memory; rows are shared out unevenly when the size does not divide 128."""
+    from paper_2605_26632_b200 import binding
+
+    monkeypatch.setenv("LYNX_PL_SPLITS", str(splits))
+    ctx = binding.Lynx(0)
+    try:
+        M, R = 390, 64
+        X = inputs.make_x(M, K, "outlier", 90 + splits)
+        _, LB = inputs.make_lora(8, K, R, 91 + splits)
+        values, meta, T = ctx.prune_compress_lora(X.cuda(), LB.cuda(), 1)
+        ov, om = oracle.compress(u16(X))
+        assert (u16(values) == ov).all()
+        assert (meta.cpu().numpy() == oracle.meta_canon_to_hw(om, M, K)).all()
+        ref = oracle_t(X, LB, 1)
+        got = T.float().cpu().numpy()
+        tol = 2.0 ** -8 * np.abs(ref) + 1e-5 * np.abs(ref).max()
+        assert (np.abs(got - ref) <= tol).all(), float(np.abs(got - ref).max())
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
+
+
+def test_prune_compress_lora_zero_rows_leading_dimensions_and_errors(lx):
+    from paper_2605_26632_b200 import binding
+
+    M, K, R = 200, 384, 64
+    X = inputs.make_x(M, K, "outlier", 9)
+    X[5] = 0
+    X[199] = 0
+    _, LB = inputs.make_lora(8, K, R, 9)
+    wideX = torch.zeros((M, K + 64), dtype=torch.bfloat16)
+    wideX[:, :K] = X
+    wideLB = torch.zeros((R, K + 8), dtype=torch.bfloat16)
+    wideLB[:, :K] = LB
+    buf = torch.full((M, 2 * R), 7.0, dtype=torch.bfloat16, device="cuda")
+    values, meta, T = lx.prune_compress_lora(wideX.cuda()[:, :K], wideLB.cuda()[:, :K], 1, T=buf[:, :R])
+    assert (T[5] == 0).all() and (T[199] == 0).all()
+    assert (buf[:, R:] == 7.0).all()
+    ov, om = oracle.compress(u16(X))
+    assert (u16(values) == ov).all()
+    assert (meta.cpu().numpy() == oracle.meta_canon_to_hw(om, M, K)).all()
+    ref = oracle_t(X, LB, 1)
+    assert np.abs(T.float().cpu().numpy() - ref).max() <= 2.0 ** -8 * np.abs(ref).max() + 1e-6
+    for bad_mode in (binding.COMP_TENSOR, binding.COMP_GROUP):
+        with pytest.raises(binding.LynxError) as e:
+            lx.prune_compress_lora(X.cuda(), LB.cuda(), bad_mode)
+        assert e.value.status == 1
+    with pytest.raises(binding.LynxError) as e:  # rank 32 is not built
+        lx.prune_compress_lora(X.cuda(), LB.cuda()[:32], 1)
+    assert e.value.status == 2
+
+
 def test_lora_down_zero_rows_and_strided_output(lx):
     M, K, R = 200, 256, 64
     X = inputs.make_x(M, K, "outlier", 7)
@@ -110,8 +201,8 @@ def test_tiny_config_with_lora_full_oracle(lx, mode, with_bias, with_res):
     cu = lambda t: None if t is None else t.cuda()
     Y = lx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), cu(b), mode, cu(res))
     check_y(Y, ref["Y"])
-    # the three-call form (own down-projection kernel; the layer call computes T inside the GEMM
-    # launch with another K split, so the two may differ in T's last bit)
+    # the three-call form (own down-projection kernel; the layer call computes T in its prune launch
+    # with another K split, so the two may differ in T's last bit)
     values, meta, scale = lx.prune_compress(X.cuda(), mode)
     T = lx.lora_down(X.cuda(), LB.cuda(), scale)
     Y2 = lx.sparse_linear_lora(values, meta, W.cuda(), T, LA.cuda(), cu(b), scale, cu(res))
@@ -148,12 +239,13 @@ def test_three_call_form_equals_unfused_layer_bit_for_bit(monkeypatch):
         ctx.close()
 
 
-@pytest.mark.parametrize("fuse", [1, 0])
+@pytest.mark.parametrize("fuse", [2, 1, 0])
 @pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6, 7])
 @pytest.mark.parametrize("R", [64, 128])
 def test_every_tile_configuration_with_lora(cfg, R, fuse, monkeypatch):
-    """fuse = 1: the down projection runs inside the GEMM launch where the tile has room for it
-    (rank 64, every tile but the 256 x 128 pair tile); fuse = 0: always as its own kernel."""
+    """fuse = 2 (default): the down projection runs in the prune launch; fuse = 1: inside the GEMM
+    launch where the tile has room for it (rank 64, every tile but the 256 x 128 pair tile);
+    fuse = 0: always as its own kernel."""
     from paper_2605_26632_b200 import binding
 
     if fuse == 0 and R == 128:
