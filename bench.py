@@ -378,8 +378,8 @@ def main():
         lora_ms = l0.elapsed_time(l1) / args.steps
         lora = {"rank": R, "ms_per_step": lora_ms, "overhead_vs_step": lora_ms / (total_ms / args.steps) - 1.0,
                 "speedup_vs_dense_bf16_without_lora": dense_ms / lora_ms,
-                "how": "lynx_act_sparse_linear_lora: prune/compress + sparse GEMM whose launch also computes "
-                       "T = (X L_B^T) / s and adds T L_A^T in its accumulator"}
+                "how": "lynx_act_sparse_linear_lora: one launch that prunes / compresses X and computes "
+                       "T = (X L_B^T) / s from the same read of X, then the sparse GEMM that adds T L_A^T in its accumulator"}
 
     # the same layer on FP8 (E4M3) operands, outside the headline number: weights quantised once
     # (symmetric per output channel), activations pruned and quantised (per-row scale found in the

@@ -1,6 +1,6 @@
 """Runs a few launches of one kernel of the path on a named synthetic workload.
 
-    python -m paper_2605_26632_b200.run_case --kernel prune|gemm|layer|fused|lora_down|lora_layer|fp8_prune|fp8_gemm|fp8_layer --workload mlp_down [--iters 3]
+    python -m paper_2605_26632_b200.run_case --kernel prune|gemm|layer|fused|lora_down|prune_lora|lora_layer|fp8_prune|fp8_gemm|fp8_layer --workload mlp_down [--iters 3]
 
 Meant as the small, self-terminating command to put under a profiler (one kernel, a few launches,
 well under a GB on the device), and as a minimal usage example of the binding.
@@ -16,7 +16,7 @@ from . import binding, inputs
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="layer", choices=["prune", "gemm", "layer", "fused", "lora_down", "lora_layer", "fp8_prune", "fp8_gemm",
+    ap.add_argument("--kernel", default="layer", choices=["prune", "gemm", "layer", "fused", "lora_down", "prune_lora", "lora_layer", "fp8_prune", "fp8_gemm",
                              "fp8_layer"])
     ap.add_argument("--rank", type=int, default=64, help="rank R of the low-rank branch")
     ap.add_argument("--workload", default="mlp_down")
@@ -39,7 +39,7 @@ def main():
     LB = (torch.randn(R, wl.K, device="cuda", generator=g) * wl.K ** -0.5).to(torch.bfloat16)
     LA = (torch.randn(wl.N, R, device="cuda", generator=g) * 0.3 * R ** -0.5).to(torch.bfloat16)
     T = torch.empty(M, R, device="cuda", dtype=torch.bfloat16)
-    if args.kernel.startswith("lora"):
+    if "lora" in args.kernel:
         lx.reserve_lora(M, wl.K, R)
     if args.kernel.startswith("fp8"):
         Wq, ws = lx.quantize_weights_fp8(W, per_channel=True)
@@ -57,6 +57,8 @@ def main():
             lx.sparse_linear(values, meta, W, b, scale, None, Y)
         if args.kernel == "lora_down":
             lx.lora_down(X, LB, scale, T)
+        if args.kernel == "prune_lora":
+            lx.prune_compress_lora(X, LB, args.comp, values, meta, T)
         if args.kernel == "lora_layer":
             lx.act_sparse_linear_lora(X, W, LA, LB, b, args.comp, None, Y)
         if args.kernel == "fused":

@@ -168,9 +168,9 @@ def fp8_sweep(lx, shapes, iters):
 
 
 def lora_sweep(lx, shapes, R, iters):
-    print("| M | K | N | R | lora_down us | lora_down GB/s | layer us | layer+LoRA us | overhead | "
+    print("| M | K | N | R | prune us | prune+down us | lora_down us | layer us | layer+LoRA us | overhead | "
           "dense+LoRA (torch) us | speedup with LoRA |")
-    print("|---|---|---|---|---|---|---|---|---|---|---|")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|")
     for (M, K, N) in shapes:
         per_set = M * K * 2 + M * K + M * K // 8 + N * K * 2 + M * N * 2
         nsets = max(2, math.ceil(400e6 / per_set))
@@ -185,6 +185,10 @@ def lora_sweep(lx, shapes, R, iters):
         ss = [torch.ones(M, device="cuda", dtype=torch.float32) for _ in range(nsets)]
         lx.reserve(M, N, K)
         lx.reserve_lora(M, K, R)
+        vs = [torch.empty(M, K // 2, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+        ms = [torch.empty(binding.meta_bytes(M, K), device="cuda", dtype=torch.uint8) for _ in range(nsets)]
+        tp = timeloop(lambda j: lx.prune_compress(Xs[j], 1, vs[j], ms[j], binding.ROW_SCALE_DEFERRED), nsets, iters)
+        tpd = timeloop(lambda j: lx.prune_compress_lora(Xs[j], LB, 1, vs[j], ms[j], Ts[j]), nsets, iters)
         td = timeloop(lambda j: lx.lora_down(Xs[j], LB, ss[j], Ts[j]), nsets, iters)
         tl = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_SEPARATE), nsets, iters)
         tll = timeloop(lambda j: lx.act_sparse_linear_lora(Xs[j], Ws[j], LA, LB, b, 1, None, Ys[j]), nsets, iters)
@@ -194,10 +198,10 @@ def lora_sweep(lx, shapes, R, iters):
             y.addmm_(torch.nn.functional.linear(Xs[j], LB), LA.t())
 
         tdl = timeloop(dense_lora, nsets, iters)
-        print(f"| {M} | {K} | {N} | {R} | {td*1e3:.1f} | {M*K*2/td/1e6:.0f} | {tl*1e3:.1f} | {tll*1e3:.1f} | "
+        print(f"| {M} | {K} | {N} | {R} | {tp*1e3:.1f} | {tpd*1e3:.1f} | {td*1e3:.1f} | {tl*1e3:.1f} | {tll*1e3:.1f} | "
               f"{100*(tll/tl-1):.1f} % | {tdl*1e3:.1f} | {tdl/tll:.2f} |", flush=True)
         assert lx.last_error() == 0
-        del Xs, Ws, Ys, Ts, ss
+        del Xs, Ws, Ys, Ts, ss, vs, ms
         torch.cuda.empty_cache()
 
 
