@@ -232,7 +232,9 @@ LYNX_API lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_ho
  *   the per-row norm compensation (mode LYNX_COMP_ROW) or 1 (LYNX_COMP_NONE; other modes:
  *   LYNX_ERR_INVALID_ARG).  Under LYNX_COMP_ROW the row sums stay on the context, exactly as
  *   after lynx_prune_compress with LYNX_ROW_SCALE_DEFERRED: pass comp->row_scale =
- *   LYNX_ROW_SCALE_DEFERRED to the lynx_sparse_linear_lora call that follows.
+ *   LYNX_ROW_SCALE_DEFERRED to the lynx_sparse_linear_lora call that follows.  Alignment: values
+ *   32-byte aligned (32-byte vector stores); X, L_B, T and meta 16-byte aligned, ldx, ldlb and ldt
+ *   multiples of 8.  Scratch: the row sums only; no low-rank workspace.
  * lynx_sparse_linear_lora:  lynx_sparse_linear plus the T L_A^T term; T must come from
  *   lynx_lora_down called with the same row_scale that comp carries, or from
  *   lynx_prune_compress_lora (deferred row scale).
