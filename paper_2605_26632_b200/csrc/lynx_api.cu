@@ -51,6 +51,7 @@ struct lynx_ctx {
     int prune_tpu = 0;  // 0 = auto
     int fp8_ring = 1;   // FP8 activations: single-read ring kernel (LYNX_FP8_RING=0: one CTA per 16 rows)
     int fp8_ring_forced = 0;
+    int gemm_group_m = 16;    // row tiles per group of the GEMM's tile order (LYNX_GEMM_GROUP_M; 0 = one group)
     int pl_force_splits = 0;  // development override: cluster size of the prune + down-projection kernel
     std::mutex mu;
 };
@@ -263,6 +264,7 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     p.dev_error = ctx->err_dev;
     p.tiles_m = (int)((M + Cfg::BM * Cfg::CG - 1) / (Cfg::BM * Cfg::CG));
     p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
+    p.group_m = (ctx->gemm_group_m > 0 && ctx->gemm_group_m < p.tiles_m) ? ctx->gemm_group_m : p.tiles_m;
     p.sk_partial = nullptr;
     p.sk_flags = nullptr;
     p.sk_epoch = 0;
@@ -419,6 +421,7 @@ lynx_status launch_gemm_fp8_cfg(lynx_ctx* ctx, const void* values_q, const void*
     p.dev_error = ctx->err_dev;
     p.tiles_m = (int)((M + Cfg::BM * Cfg::CG - 1) / (Cfg::BM * Cfg::CG));
     p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
+    p.group_m = (ctx->gemm_group_m > 0 && ctx->gemm_group_m < p.tiles_m) ? ctx->gemm_group_m : p.tiles_m;
     p.l0_splits = 1;
     auto kern = sparse_gemm_kernel<Cfg, false>;
     static bool attr_set[MAX_CTX_DEVICES] = {};  // per instantiation
@@ -757,6 +760,8 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
     if (env) ctx->defer_scale = atoi(env);
     env = getenv("LYNX_PRUNE_TPU");  // development override: 128-element K blocks per warp
     if (env) ctx->prune_tpu = atoi(env);
+    env = getenv("LYNX_GEMM_GROUP_M");  // development override: row tiles per group of the GEMM's tile order
+    if (env) ctx->gemm_group_m = atoi(env);
     env = getenv("LYNX_PL_SPLITS");  // development override: K splits (= cluster size) of the prune + down-projection kernel
     if (env) ctx->pl_force_splits = atoi(env);
     env = getenv("LYNX_FP8_RING");  // development override: 0 = one CTA per 16 rows, n = ring with n warps per row

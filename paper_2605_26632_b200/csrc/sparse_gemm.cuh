@@ -53,6 +53,7 @@ struct GemmParams {
     int64_t ldr;
     uint32_t* dev_error;  // sticky error word (host-visible)
     int tiles_m, tiles_n;
+    int group_m;  // tile order: groups of `group_m` row tiles are swept over all of N before the next group
     // stream-K tail (see TileSchedule): fp32 partial tiles, one slot per cluster, and one ready
     // word per (slot, epilogue warp of the pair) holding the launch epoch; nullptr = off
     float* sk_partial;
@@ -85,6 +86,18 @@ struct WorkItem {
     int kind;           // 0 whole tile, 1 partial piece (write fp32), 2 owner piece (add partials)
     int first_contrib;  // owner: clusters first_contrib .. c-1 hold the partials
 };
+// Tile index -> (row tile, column tile).  Inside a group of `group_m` row tiles the row index runs
+// fastest, the groups follow one another: the tiles that run at the same time then share
+// group_m blocks of A and tiles / group_m blocks of W, whatever M is (with one group over all of
+// M a wave of a tall problem would stream the whole of A from HBM once per column tile).
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int group_m, int& tm, int& tn) {
+    const int per_group = group_m * tiles_n;
+    const int g = tile / per_group, r = tile - g * per_group;
+    const int rows = (tiles_m - g * group_m < group_m) ? tiles_m - g * group_m : group_m;
+    tn = r / rows;
+    tm = g * group_m + (r - tn * rows);
+}
+
 struct TileSchedule {
     int T, C, KB, full, R, total;
     bool streamk;
@@ -351,7 +364,8 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             }
             for (int wi = 0; wi < num_items && ok; ++wi) {
                 const WorkItem w = sched.get(cluster_id, wi);
-                const int tm = w.tile % p.tiles_m, tn = w.tile / p.tiles_m;
+                int tm, tn;
+                tile_coords(w.tile, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
                 const int m0 = (tm * CG + (int)rank) * Cfg::BM;
                 const int n0 = tn * BN + (int)rank * Cfg::BN_CTA;
                 const int eblk = (tm * CG + (int)rank) * kblocks;
@@ -657,7 +671,8 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         }
         for (; it < num_items && alive; ++it) {
             const WorkItem w = sched.get(cluster_id, it);
-            const int tm = w.tile % p.tiles_m, tn = w.tile / p.tiles_m;
+            int tm, tn;
+            tile_coords(w.tile, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
             const int gi = l0_n + it;
             const int acc = (Cfg::ACC_STAGES == 2) ? (gi & 1) : 0;
             const uint32_t acc_phase = (Cfg::ACC_STAGES == 2) ? ((gi >> 1) & 1) : (gi & 1);
