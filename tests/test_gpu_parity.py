@@ -508,4 +508,16 @@ def test_argument_errors_are_reported_not_launched(lx):
                                          c_void_p(values.data_ptr()), c_void_p(meta.data_ptr()), None, 1, None)
         binding._check(st, "prune")
     assert e.value.status == 1
+    # an empty problem (M = 0) is refused by every entry point before anything is launched
+    from ctypes import c_void_p
+    n0 = lx.launch_count()
+    vp, mp = c_void_p(values.data_ptr()), c_void_p(meta.data_ptr())
+    Wk = torch.zeros(16, 128, dtype=torch.bfloat16, device="cuda")
+    Y = torch.zeros(16, 16, dtype=torch.bfloat16, device="cuda")
+    wp, yp = c_void_p(Wk.data_ptr()), c_void_p(Y.data_ptr())
+    assert lx._lib.lynx_prune_compress(lx._h, vp, 0, 128, 128, vp, mp, None, 0, None) == 1
+    assert lx._lib.lynx_sparse_linear(lx._h, vp, mp, 0, 128, wp, 16, 128, None, None, yp, 16, None) == 1
+    assert lx._lib.lynx_act_sparse_linear(lx._h, vp, 0, 128, 128, wp, 16, 128, None, 0, None, 0, yp, 16, 0, None) == 1
+    assert lx._lib.lynx_prune_compress_fp8(lx._h, vp, 0, 256, 256, None, vp, mp, c_void_p(Y.data_ptr()), 0, None) == 1
+    assert lx.launch_count() == n0
     assert lx.last_error() == 0
