@@ -213,6 +213,15 @@ ScratchLayout scratch_layout(int64_t M, int64_t N, int64_t K) {
 
 // --------------------------------------------------------------------------- GEMM launch -----
 
+// Row tiles per group of the GEMM's tile order: groups of about `gemm_group_m` (16), all of nearly the
+// same size (17 row tiles run as 9 + 8, not as 16 + 1: a one-row group shares no W tile between clusters).
+static int gemm_group_rows(const lynx_ctx* ctx, int tiles_m) {
+    const int g = ctx->gemm_group_m;
+    if (g <= 0 || g >= tiles_m) return tiles_m;
+    const int groups = (tiles_m + g - 1) / g;
+    return (tiles_m + groups - 1) / groups;
+}
+
 template <class Cfg>
 lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
                             const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
@@ -264,7 +273,7 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     p.dev_error = ctx->err_dev;
     p.tiles_m = (int)((M + Cfg::BM * Cfg::CG - 1) / (Cfg::BM * Cfg::CG));
     p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
-    p.group_m = (ctx->gemm_group_m > 0 && ctx->gemm_group_m < p.tiles_m) ? ctx->gemm_group_m : p.tiles_m;
+    p.group_m = gemm_group_rows(ctx, p.tiles_m);
     p.sk_partial = nullptr;
     p.sk_flags = nullptr;
     p.sk_epoch = 0;
@@ -421,7 +430,7 @@ lynx_status launch_gemm_fp8_cfg(lynx_ctx* ctx, const void* values_q, const void*
     p.dev_error = ctx->err_dev;
     p.tiles_m = (int)((M + Cfg::BM * Cfg::CG - 1) / (Cfg::BM * Cfg::CG));
     p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
-    p.group_m = (ctx->gemm_group_m > 0 && ctx->gemm_group_m < p.tiles_m) ? ctx->gemm_group_m : p.tiles_m;
+    p.group_m = gemm_group_rows(ctx, p.tiles_m);
     p.l0_splits = 1;
     auto kern = sparse_gemm_kernel<Cfg, false>;
     static bool attr_set[MAX_CTX_DEVICES] = {};  // per instantiation
