@@ -77,8 +77,11 @@ typedef enum {
  * at its per-K-split row sums, kept in the context, instead of finishing s_m itself (which costs a
  * hand-over between its CTAs); pass it as comp->row_scale to the lynx_sparse_linear call that
  * follows ON THE SAME CONTEXT with the same M and K, and its epilogue forms s_m from those sums,
- * in the same order of additions (same bits).  A later lynx_prune_compress or layer call on the
- * context overwrites the sums. */
+ * in the same order of additions (same bits).  The sums live in the context's scratch: any later
+ * call on the context that writes the scratch (another lynx_prune_compress in ROW / TENSOR mode,
+ * any lynx_act_sparse_linear* call) or regrows it (lynx_reserve, a larger shape) makes the context
+ * forget them, and a lynx_sparse_linear call that still asks for them returns
+ * LYNX_ERR_INVALID_ARG without launching anything. */
 #define LYNX_ROW_SCALE_DEFERRED ((float*)(uintptr_t)1)
 
 /* Epilogue terms of lynx_sparse_linear (all optional). */
@@ -91,7 +94,11 @@ typedef struct {
 /* ---- context ------------------------------------------------------------------------------- */
 
 /* Creates a context on CUDA device `device` (made current for the call).  Allocates a small
- * status word; scratch is allocated lazily (see lynx_reserve).  */
+ * status word and a ticket area; scratch is allocated lazily (see lynx_reserve).  The context
+ * caches the tensor maps (TMA descriptors) it encodes, keyed by pointer, shape, leading dimension
+ * and tile, so a layer called again on the same buffers re-encodes nothing.  Reads no environment
+ * variable except LYNX_DEV: with LYNX_DEV=1 (tests, measurement scripts) it also reads the
+ * development overrides (LYNX_GEMM_CFG, LYNX_SPLITK, LYNX_PRUNE_TPU, ...). */
 LYNX_API lynx_status lynx_create(lynx_ctx** out, int device);
 /* Frees the context's scratch.  The caller must have synchronised every stream it used. */
 LYNX_API lynx_status lynx_destroy(lynx_ctx* ctx);
@@ -103,7 +110,8 @@ LYNX_API lynx_status lynx_last_error(lynx_ctx* ctx);
 /* Bytes of the compressed operands for an M x K activation matrix. */
 LYNX_API size_t lynx_values_bytes(int64_t M, int64_t K); /* M * (K/2) bf16                    */
 LYNX_API size_t lynx_meta_bytes(int64_t M, int64_t K);   /* ceil(M/128) * (K/128) * 2048      */
-/* Scratch the context needs for lynx_act_sparse_linear / TENSOR compensation at this size. */
+/* Scratch the context needs for lynx_act_sparse_linear / TENSOR compensation at this size
+ * (partial row sums, compressed operands, row scale; N does not enter). */
 LYNX_API size_t lynx_workspace_bytes(int64_t M, int64_t N, int64_t K);
 /* Grows the context's scratch to serve shapes up to (M, N, K).  May call cudaMalloc and
  * synchronise; call it outside timed or captured regions.  Entry points that need scratch call
@@ -164,7 +172,8 @@ LYNX_API lynx_status lynx_prune_compress(lynx_ctx* ctx, const void* X, int64_t M
  *     calls that overlap on the GPU (different streams, no ordering between them) race on it:
  *     order them.
  *   - No device-side error word: the kernels involved have no waits that can time out.
- * Arguments, layouts, alignment rules and results are exactly those of lynx_prune_compress. */
+ * Arguments, layouts, alignment rules and results are exactly those of lynx_prune_compress (one
+ * work decomposition serves both, so row_scale agrees bit for bit). */
 #define LYNX_STATIC_SCRATCH_BYTES (8u << 20)
 LYNX_API lynx_status lynx_prune_compress_static(const void* X, int64_t M, int64_t K, int64_t ldx,
                                                 void* values, void* meta, float* row_scale,
@@ -201,7 +210,8 @@ LYNX_API lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_
 /* Same layer with the activations and the result in HOST memory (pinned memory recommended):
  * X_host [M x K] and Y_host [M x N] are dense row-major bf16 HOST buffers; W and bias stay
  * DEVICE resident (weights are loaded once).  Copies X to the device, runs the layer, copies Y
- * back and synchronises `stream`.  Staging buffers live in the context's scratch.  From 2048 rows
+ * back and synchronises `stream`.  The device mirrors of X and Y are an allocation of their own that
+ * only this entry point makes (grown on demand, like the scratch).  From 2048 rows
  * on (and not under LYNX_COMP_TENSOR, whose scale couples all rows) the call is pipelined over row
  * chunks on two copy streams the context owns, so that copy-in, kernels and copy-out overlap; the
  * result is the unchunked one bit for bit. */

@@ -24,8 +24,10 @@ struct lynx_ctx {
     int num_sms = 0;
     uint32_t* err_host = nullptr;  // mapped pinned word written by kernels
     uint32_t* err_dev = nullptr;
-    void* scratch = nullptr;  // compressed operands, scale, sums, host staging mirrors
+    void* scratch = nullptr;  // partial row sums, compressed operands and scale of the single-call path
     size_t scratch_bytes = 0;
+    void* host_stage = nullptr;  // device mirrors of X and Y, only for lynx_act_sparse_linear_host
+    size_t host_stage_bytes = 0;
     uint32_t* tickets = nullptr;  // one word per 16-row block (prune finalize), zero between launches
     void* lora_ws = nullptr;      // low-rank branch: [fp32 partials][T]
     size_t lora_ws_bytes = 0;
@@ -53,6 +55,25 @@ struct lynx_ctx {
     int fp8_ring_forced = 0;
     int gemm_group_m = 16;    // row tiles per group of the GEMM's tile order (LYNX_GEMM_GROUP_M; 0 = one group)
     int pl_force_splits = 0;  // development override: cluster size of the prune + down-projection kernel
+    int splitk_force = 1;     // in-cluster split-K of the GEMM for launches with few tiles: 1 = cost model, 0 = off, 2..4 forced
+    int prune_finalize = 0;   // row-scale finalize of the stand-alone prune call: 0 = per shape, 1 = in-kernel ticket, 2 = own launch
+    // encoded tensor maps of recent launches, keyed by everything that went into the encoding
+    // (a layer called again on the same buffers skips cuTensorMapEncodeTiled)
+    struct TmapKey {
+        const void* base;
+        uint64_t rows, cols, ld_bytes;
+        uint32_t box_cols, box_rows;
+        int dt, sw;
+        bool operator==(const TmapKey& o) const {
+            return base == o.base && rows == o.rows && cols == o.cols && ld_bytes == o.ld_bytes &&
+                   box_cols == o.box_cols && box_rows == o.box_rows && dt == o.dt && sw == o.sw;
+        }
+    };
+    static constexpr int TMAP_CACHE = 128;  // direct mapped
+    TmapKey tmap_key[TMAP_CACHE] = {};
+    CUtensorMap tmap_val[TMAP_CACHE];
+    bool tmap_ok[TMAP_CACHE] = {};
+    int64_t tmap_hits = 0, tmap_misses = 0;
     std::mutex mu;
 };
 
@@ -77,18 +98,40 @@ EncodeTiledFn get_encode() {
 }
 
 // 2D row-major tensor [rows x cols] of `elem_bytes` elements, row pitch `ld_bytes`.
-bool make_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t rows,
-                  uint64_t cols, uint64_t ld_bytes, uint32_t box_cols, uint32_t box_rows,
-                  CUtensorMapSwizzle sw) {
+bool encode_tmap_2d(CUtensorMap* m, CUtensorMapDataType dt, const void* base, uint64_t rows, uint64_t cols,
+                    uint64_t ld_bytes, uint32_t box_cols, uint32_t box_rows, CUtensorMapSwizzle sw) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {ld_bytes};
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    (void)elem_bytes;
     return enc(m, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The same through the context's cache: a tensor map is a pure function of its key, so a hit is
+// exact.  (One context serves one stream at a time; the cache is not locked.)
+bool make_tmap_2d(lynx_ctx* ctx, CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const void* base,
+                  uint64_t rows, uint64_t cols, uint64_t ld_bytes, uint32_t box_cols, uint32_t box_rows,
+                  CUtensorMapSwizzle sw) {
+    (void)elem_bytes;
+    const lynx_ctx::TmapKey key{base, rows, cols, ld_bytes, box_cols, box_rows, (int)dt, (int)sw};
+    uint64_t h = reinterpret_cast<uintptr_t>(base) >> 8;
+    h = h * 0x9E3779B97F4A7C15ull + rows * 31 + cols * 131 + ld_bytes * 7 + box_cols * 1009 + box_rows * 9176 +
+        (uint64_t)dt * 77 + (uint64_t)sw;
+    const int slot = (int)((h >> 20) % lynx_ctx::TMAP_CACHE);
+    if (ctx->tmap_ok[slot] && ctx->tmap_key[slot] == key) {
+        *m = ctx->tmap_val[slot];
+        ctx->tmap_hits++;
+        return true;
+    }
+    if (!encode_tmap_2d(m, dt, base, rows, cols, ld_bytes, box_cols, box_rows, sw)) return false;
+    ctx->tmap_key[slot] = key;
+    ctx->tmap_val[slot] = *m;
+    ctx->tmap_ok[slot] = true;
+    ctx->tmap_misses++;
+    return true;
 }
 
 // cudaFuncSetAttribute is per device: remember, per kernel instantiation, which devices have it.
@@ -188,14 +231,15 @@ L0Plan l0_plan(int clusters, int tiles, int tiles_m, int kblocks, double t_tile_
 // upper bound of the splits any plan uses (workspace sizing)
 constexpr int L0_MAX_SPLITS = 16;
 
-// Scratch layout for (M, N, K):
-// [partial row sums][sums 2M floats][values][meta][row_scale M floats][X stage][Y stage]
+// Scratch layout for (M, K):
+// [partial row sums][sums 2M floats][values][meta][row_scale M floats]
 // The first two sections serve lynx_prune_compress alone and come first so that a context that is
-// only used for pruning needs little memory.
+// only used for pruning needs little memory.  (The device mirrors of host buffers belong to
+// lynx_act_sparse_linear_host alone and live in an allocation of their own.)
 struct ScratchLayout {
-    size_t partial, prune_end, values, meta, scale, sums, xstage, ystage, total;
+    size_t partial, prune_end, values, meta, scale, sums, total;
 };
-ScratchLayout scratch_layout(int64_t M, int64_t N, int64_t K) {
+ScratchLayout scratch_layout(int64_t M, int64_t K) {
     ScratchLayout L;
     size_t off = 0;
     const size_t rb16 = (size_t)((M + 127) / 128) * 8, kblocks = (size_t)(K / 128);
@@ -205,10 +249,35 @@ ScratchLayout scratch_layout(int64_t M, int64_t N, int64_t K) {
     L.values = off; off = align_up(off + lynx_values_bytes(M, K), 1024);
     L.meta = off;   off = align_up(off + lynx_meta_bytes(M, K), 1024);
     L.scale = off;  off = align_up(off + (size_t)M * 4, 1024);
-    L.xstage = off; off = align_up(off + (size_t)M * K * 2, 1024);
-    L.ystage = off; off = align_up(off + (size_t)M * N * 2, 1024);
     L.total = off;
     return L;
+}
+
+// Work decomposition of the prune/compress launch: one warp per (16-row block, run of `tpu`
+// 128-element K blocks), KS = runs per row, 4 warps per CTA.  Shared by every entry point that
+// launches prune_compress_kernel: the bits of the row sums depend on KS.
+struct PrunePlan {
+    int64_t rb16;
+    int tpu, KS, ctas_per_rb;
+    unsigned grid;
+};
+PrunePlan prune_plan(int num_sms, int64_t M, int64_t K, int tpu_override) {
+    PrunePlan P;
+    const int64_t kblocks = K / 128;
+    P.rb16 = ((M + 127) / 128) * 8;
+    int tpu = tpu_override;
+    if (tpu <= 0) {
+        const int64_t resident = (int64_t)num_sms * 40;  // warps the GPU holds at ~48 registers
+        const int64_t want = (P.rb16 * kblocks) / (3 * resident);
+        tpu = (int)(want < 1 ? 1 : (want > 8 ? 8 : want));
+    }
+    if (tpu > kblocks) tpu = (int)kblocks;
+    while (kblocks % tpu) --tpu;
+    P.tpu = tpu;
+    P.KS = (int)(kblocks / tpu);
+    P.ctas_per_rb = (P.KS + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS;
+    P.grid = (unsigned)(P.rb16 * P.ctas_per_rb);
+    return P;
 }
 
 // --------------------------------------------------------------------------- GEMM launch -----
@@ -228,19 +297,19 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
                             const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st, const ScaleSrc* ss) {
     CUtensorMap ta, tb, te, ty, tt, tla, tx, tlb;
     const uint64_t rb = (uint64_t)((M + 127) / 128), kblocks = (uint64_t)(K / 128);
-    if (!make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, values, (uint64_t)M, (uint64_t)(K / 2),
+    if (!make_tmap_2d(ctx, &ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, values, (uint64_t)M, (uint64_t)(K / 2),
                       (uint64_t)K, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)N, (uint64_t)K, (uint64_t)ldw * 2, 64,
+        !make_tmap_2d(ctx, &tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)N, (uint64_t)K, (uint64_t)ldw * 2, 64,
                       Cfg::BN_CTA, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&te, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, meta, rb * kblocks * 2, 256, 1024, 256, 2,
+        !make_tmap_2d(ctx, &te, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, meta, rb * kblocks * 2, 256, 1024, 256, 2,
                       CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, Cfg::CH,
+        !make_tmap_2d(ctx, &ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, Cfg::CH,
                       32, Cfg::CH == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE))
         return LYNX_ERR_CUDA;
     if (lora) {
-        if (!make_tmap_2d(&tt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->T, (uint64_t)M, (uint64_t)lora->R,
+        if (!make_tmap_2d(ctx, &tt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->T, (uint64_t)M, (uint64_t)lora->R,
                           (uint64_t)lora->ldt * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap_2d(&tla, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->LA, (uint64_t)N, (uint64_t)lora->R,
+            !make_tmap_2d(ctx, &tla, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->LA, (uint64_t)N, (uint64_t)lora->R,
                           (uint64_t)lora->ldla * 2, 64, Cfg::BN_CTA, CU_TENSOR_MAP_SWIZZLE_128B))
             return LYNX_ERR_CUDA;
     } else {
@@ -250,9 +319,9 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     const bool l0 = lora && lora->X && Cfg::L0_OK && lora->R == Cfg::L0_R;
     if (lora && lora->X && !l0) return LYNX_ERR_INVALID_ARG;  // the caller checks the tile first
     if (l0) {
-        if (!make_tmap_2d(&tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->X, (uint64_t)M, (uint64_t)K,
+        if (!make_tmap_2d(ctx, &tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->X, (uint64_t)M, (uint64_t)K,
                           (uint64_t)lora->ldx * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap_2d(&tlb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->LB, (uint64_t)lora->R, (uint64_t)K,
+            !make_tmap_2d(ctx, &tlb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->LB, (uint64_t)lora->R, (uint64_t)K,
                           (uint64_t)lora->ldlb * 2, 64, Cfg::L0_R / Cfg::CG, CU_TENSOR_MAP_SWIZZLE_128B))
             return LYNX_ERR_CUDA;
     } else {
@@ -303,14 +372,7 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
         const int kblocks = (int)(K / Cfg::BK);
         const int rem = tiles % clusters;
         if (!l0 && ctx->streamk && rem > 0 && (int64_t)rem * kblocks >= 4ll * clusters) {
-            if (!ctx->sk_partial) {
-                const size_t slot = (size_t)128 * 256 * 4, nslots = (size_t)ctx->num_sms;
-                void* buf = nullptr;
-                if (cudaMalloc(&buf, nslots * slot + nslots * 8 * 4) != cudaSuccess) return LYNX_ERR_WORKSPACE;
-                if (cudaMemset(buf, 0, nslots * slot + nslots * 8 * 4) != cudaSuccess) return LYNX_ERR_CUDA;
-                ctx->sk_partial = static_cast<float*>(buf);
-                ctx->sk_flags = reinterpret_cast<uint32_t*>(static_cast<char*>(buf) + nslots * slot);
-            }
+            if (!ctx->sk_partial) return LYNX_ERR_WORKSPACE;  // allocated by lynx_create when the schedule is on
             p.sk_partial = ctx->sk_partial;
             p.sk_flags = ctx->sk_flags;
             p.sk_epoch = ++ctx->sk_epoch;
@@ -411,13 +473,13 @@ lynx_status launch_gemm_fp8_cfg(lynx_ctx* ctx, const void* values_q, const void*
     static_assert(Cfg::FP8, "FP8 configuration expected");
     CUtensorMap ta, tb, te, ty;
     const uint64_t rb = (uint64_t)((M + 127) / 128), kb128 = (uint64_t)(K / 128);
-    if (!make_tmap_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, values_q, (uint64_t)M, (uint64_t)(K / 2),
+    if (!make_tmap_2d(ctx, &ta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, values_q, (uint64_t)M, (uint64_t)(K / 2),
                       (uint64_t)(K / 2), 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldwq, 128,
+        !make_tmap_2d(ctx, &tb, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldwq, 128,
                       Cfg::BN_CTA, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&te, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, meta, rb * kb128 * 2, 256, 1024, 256,
+        !make_tmap_2d(ctx, &te, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, meta, rb * kb128 * 2, 256, 1024, 256,
                       Cfg::E_BYTES / 1024, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, Cfg::CH,
+        !make_tmap_2d(ctx, &ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, Cfg::CH,
                       32, Cfg::CH == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE))
         return LYNX_ERR_CUDA;
     GemmParams p = {};
@@ -482,11 +544,11 @@ lynx_status launch_fused(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int
                          int64_t ldy, cudaStream_t st) {
     using Cfg = FusedCfg;
     CUtensorMap tx, tb, ty;
-    if (!make_tmap_2d(&tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx * 2, 64,
+    if (!make_tmap_2d(ctx, &tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx * 2, 64,
                       Cfg::BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)N, (uint64_t)K, (uint64_t)ldw * 2, 64,
+        !make_tmap_2d(ctx, &tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)N, (uint64_t)K, (uint64_t)ldw * 2, 64,
                       Cfg::BN, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, 64,
+        !make_tmap_2d(ctx, &ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, 64,
                       32, CU_TENSOR_MAP_SWIZZLE_128B))
         return LYNX_ERR_CUDA;
     FusedParams p;
@@ -517,14 +579,36 @@ lynx_status check_common(lynx_ctx* ctx, int64_t M, int64_t K) {
     return LYNX_OK;
 }
 
+// The deferred row sums of a two-call user live in the scratch: whoever reallocates it or writes
+// other data into it forgets them, so that a GEMM call that still asks for them is refused
+// (LYNX_ERR_INVALID_ARG) instead of reading freed or overwritten memory.
+void clear_deferred(lynx_ctx* ctx) {
+    ctx->deferred_partial = nullptr;
+    ctx->deferred_ks = 0;
+    ctx->deferred_M = 0;
+    ctx->deferred_K = 0;
+}
+
 lynx_status ensure_scratch(lynx_ctx* ctx, size_t bytes) {
     if (ctx->scratch_bytes >= bytes) return LYNX_OK;
+    clear_deferred(ctx);
     if (cudaDeviceSynchronize() != cudaSuccess) return LYNX_ERR_CUDA;
     if (ctx->scratch) cudaFree(ctx->scratch);
     ctx->scratch = nullptr;
     ctx->scratch_bytes = 0;
     if (cudaMalloc(&ctx->scratch, bytes) != cudaSuccess) return LYNX_ERR_WORKSPACE;
     ctx->scratch_bytes = bytes;
+    return LYNX_OK;
+}
+
+lynx_status ensure_host_stage(lynx_ctx* ctx, size_t bytes) {
+    if (ctx->host_stage_bytes >= bytes) return LYNX_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) return LYNX_ERR_CUDA;
+    if (ctx->host_stage) cudaFree(ctx->host_stage);
+    ctx->host_stage = nullptr;
+    ctx->host_stage_bytes = 0;
+    if (cudaMalloc(&ctx->host_stage, bytes) != cudaSuccess) return LYNX_ERR_WORKSPACE;
+    ctx->host_stage_bytes = bytes;
     return LYNX_OK;
 }
 
@@ -587,9 +671,9 @@ lynx_status launch_lora_down(lynx_ctx* ctx, const void* X, int64_t M, int64_t K,
                              int64_t ldlb, const float* row_scale, void* T, int64_t ldt, float* partial,
                              cudaStream_t st) {
     CUtensorMap tx, tlb;
-    if (!make_tmap_2d(&tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx * 2, 64,
+    if (!make_tmap_2d(ctx, &tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx * 2, 64,
                       Cfg::BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&tlb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, LB, (uint64_t)Cfg::R, (uint64_t)K,
+        !make_tmap_2d(ctx, &tlb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, LB, (uint64_t)Cfg::R, (uint64_t)K,
                       (uint64_t)ldlb * 2, 64, Cfg::R, CU_TENSOR_MAP_SWIZZLE_128B))
         return LYNX_ERR_CUDA;
     LoraDownParams p;
@@ -645,9 +729,9 @@ lynx_status launch_prune_lora(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
                               int64_t ldlb, void* values, void* meta, float* scale_partial, void* T, int64_t ldt,
                               cudaStream_t st, int* splits_out) {
     CUtensorMap tx, tlb;
-    if (!make_tmap_2d(&tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx * 2, 64,
+    if (!make_tmap_2d(ctx, &tx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx * 2, 64,
                       Cfg::BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&tlb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, LB, (uint64_t)Cfg::R, (uint64_t)K,
+        !make_tmap_2d(ctx, &tlb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, LB, (uint64_t)Cfg::R, (uint64_t)K,
                       (uint64_t)ldlb * 2, 64, Cfg::R, CU_TENSOR_MAP_SWIZZLE_128B))
         return LYNX_ERR_CUDA;
     auto kern = prune_lora_kernel<Cfg, SUMS>;
@@ -674,9 +758,6 @@ lynx_status launch_prune_lora(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
             cap[i] = n * (i + 1);
         }
         if (cap[0] <= 0) cap[0] = ctx->num_sms;
-        if (getenv("LYNX_DEBUG_PLAN"))
-            fprintf(stderr, "prune+down: CTAs resident by cluster size 1..8: %d %d %d %d %d %d %d %d\n", cap[0], cap[1],
-                    cap[2], cap[3], cap[4], cap[5], cap[6], cap[7]);
     }
     PruneLoraParams p;
     p.M = M; p.K = K;
@@ -753,30 +834,44 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
         delete ctx;
         return LYNX_ERR_WORKSPACE;
     }
-    const char* env = getenv("LYNX_GEMM_CFG");  // development override of the tile configuration
-    if (env) ctx->gemm_cfg = atoi(env);
-    env = getenv("LYNX_PDL");  // 0 turns programmatic dependent launch off
-    if (env) ctx->pdl = atoi(env);
-    env = getenv("LYNX_STREAMK");  // 1 turns the stream-K tail on
-    if (env) ctx->streamk = atoi(env);
-    env = getenv("LYNX_LORA_FUSE");  // down projection of the low-rank branch: 0 own kernel, 1 in the GEMM launch, 2 in the prune launch
-    if (env) ctx->lora_fuse = atoi(env);
-    env = getenv("LYNX_L0_SPLITS");  // development overrides: K splits of the in-GEMM down projection,
-    if (env) ctx->l0_force_splits = atoi(env);
-    env = getenv("LYNX_L0_FILL");  // and items per light cluster (0: round-robin over all clusters)
-    if (env) ctx->l0_force_fill = atoi(env);
-    env = getenv("LYNX_DEFER_SCALE");
-    if (env) ctx->defer_scale = atoi(env);
-    env = getenv("LYNX_PRUNE_TPU");  // development override: 128-element K blocks per warp
-    if (env) ctx->prune_tpu = atoi(env);
-    env = getenv("LYNX_GEMM_GROUP_M");  // development override: row tiles per group of the GEMM's tile order
-    if (env) ctx->gemm_group_m = atoi(env);
-    env = getenv("LYNX_PL_SPLITS");  // development override: K splits (= cluster size) of the prune + down-projection kernel
-    if (env) ctx->pl_force_splits = atoi(env);
-    env = getenv("LYNX_FP8_RING");  // development override: 0 = one CTA per 16 rows, n = ring with n warps per row
-    if (env) {
-        ctx->fp8_ring = atoi(env);
-        ctx->fp8_ring_forced = 1;
+    // Development overrides (tile configuration, schedules, kernel forms) are read only when
+    // LYNX_DEV=1 is set: tests and measurement scripts set it, a production process reads nothing else.
+    const char* dev = getenv("LYNX_DEV");
+    if (dev && atoi(dev) == 1) {
+        auto geti = [](const char* name, int* dst) {
+            const char* e = getenv(name);
+            if (e) *dst = atoi(e);
+            return e != nullptr;
+        };
+        geti("LYNX_GEMM_CFG", &ctx->gemm_cfg);            // tile configuration
+        geti("LYNX_PDL", &ctx->pdl);                      // 0 turns programmatic dependent launch off
+        geti("LYNX_STREAMK", &ctx->streamk);              // 1 turns the stream-K tail on
+        geti("LYNX_LORA_FUSE", &ctx->lora_fuse);          // down projection: 0 own kernel, 1 in the GEMM launch, 2 in the prune launch
+        geti("LYNX_L0_SPLITS", &ctx->l0_force_splits);    // K splits of the in-GEMM down projection,
+        geti("LYNX_L0_FILL", &ctx->l0_force_fill);        // and items per light cluster (0: round-robin over all clusters)
+        geti("LYNX_DEFER_SCALE", &ctx->defer_scale);
+        geti("LYNX_PRUNE_TPU", &ctx->prune_tpu);          // 128-element K blocks per warp
+        geti("LYNX_GEMM_GROUP_M", &ctx->gemm_group_m);    // row tiles per group of the GEMM's tile order
+        geti("LYNX_PL_SPLITS", &ctx->pl_force_splits);    // K splits (= cluster size) of the prune + down-projection kernel
+        if (geti("LYNX_FP8_RING", &ctx->fp8_ring)) ctx->fp8_ring_forced = 1;  // 0 = one CTA per 16 rows, n = ring with n warps per row
+        geti("LYNX_SPLITK", &ctx->splitk_force);          // in-cluster split-K of the GEMM: 0 off, 1 model (default), 2..4 forced
+        geti("LYNX_PRUNE_FINALIZE", &ctx->prune_finalize);  // row-scale finalize: 0 model, 1 in-kernel ticket, 2 own launch
+    }
+    if (ctx->streamk) {
+        // stream-K partial tiles (one slot per cluster) and their ready words: allocated here so
+        // that no launch call ever allocates
+        const size_t slot = (size_t)128 * 256 * 4, nslots = (size_t)ctx->num_sms;
+        void* buf = nullptr;
+        if (cudaMalloc(&buf, nslots * slot + nslots * 8 * 4) != cudaSuccess ||
+            cudaMemset(buf, 0, nslots * slot + nslots * 8 * 4) != cudaSuccess) {
+            if (buf) cudaFree(buf);
+            cudaFree(ctx->tickets);
+            cudaFreeHost(ctx->err_host);
+            delete ctx;
+            return LYNX_ERR_WORKSPACE;
+        }
+        ctx->sk_partial = static_cast<float*>(buf);
+        ctx->sk_flags = reinterpret_cast<uint32_t*>(static_cast<char*>(buf) + nslots * slot);
     }
     *out = ctx;
     return LYNX_OK;
@@ -786,6 +881,7 @@ lynx_status lynx_destroy(lynx_ctx* ctx) {
     if (!ctx) return LYNX_ERR_INVALID_ARG;
     cudaSetDevice(ctx->device);
     if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->host_stage) cudaFree(ctx->host_stage);
     if (ctx->sk_partial) cudaFree(ctx->sk_partial);
     if (ctx->tickets) cudaFree(ctx->tickets);
     if (ctx->lora_ws) cudaFree(ctx->lora_ws);
@@ -807,7 +903,7 @@ const char* lynx_status_string(lynx_status s) {
         case LYNX_ERR_INVALID_ARG: return "invalid argument";
         case LYNX_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (need K % 128 == 0, N % 8 == 0)";
         case LYNX_ERR_ALIGNMENT: return "pointer or leading dimension not 16-byte aligned";
-        case LYNX_ERR_WORKSPACE: return "scratch allocation failed";
+        case LYNX_ERR_WORKSPACE: return "scratch too small or its allocation failed";
         case LYNX_ERR_CUDA: return "CUDA runtime error";
         case LYNX_ERR_TIMEOUT: return "device-side wait timed out";
         case LYNX_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
@@ -824,12 +920,12 @@ lynx_status lynx_last_error(lynx_ctx* ctx) {
 
 size_t lynx_values_bytes(int64_t M, int64_t K) { return (size_t)M * (size_t)(K / 2) * 2; }
 size_t lynx_meta_bytes(int64_t M, int64_t K) { return (size_t)((M + 127) / 128) * (size_t)(K / 128) * 2048; }
-size_t lynx_workspace_bytes(int64_t M, int64_t N, int64_t K) { return scratch_layout(M, N, K).total; }
+size_t lynx_workspace_bytes(int64_t M, int64_t N, int64_t K) { return scratch_layout(M, K).total; }
 
 lynx_status lynx_reserve(lynx_ctx* ctx, int64_t M, int64_t N, int64_t K) {
     if (!ctx || M < 1 || N < 1 || K < 1) return LYNX_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lock(ctx->mu);
-    return ensure_scratch(ctx, scratch_layout(M, N, K).total);
+    return ensure_scratch(ctx, scratch_layout(M, K).total);
 }
 
 int64_t lynx_launch_count(lynx_ctx* ctx) { return ctx ? ctx->launches : -1; }
@@ -855,22 +951,16 @@ static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
         return LYNX_ERR_ALIGNMENT;  // 32-byte vector accesses
     if ((s = check_device_error(ctx)) != LYNX_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // work decomposition: one warp per (16-row block, run of `tpu` K blocks)
-    const int64_t kblocks = K / 128;
-    const int64_t rb16 = ((M + 127) / 128) * 8;
-    int tpu = ctx->prune_tpu;
-    if (tpu <= 0) {
-        const int64_t resident = (int64_t)ctx->num_sms * 40;  // warps the GPU holds at ~48 registers
-        const int64_t want = (rb16 * kblocks) / (3 * resident);
-        tpu = (int)(want < 1 ? 1 : (want > 8 ? 8 : want));
-    }
-    while (kblocks % tpu) --tpu;
-    const int KS = (int)(kblocks / tpu);
+    const PrunePlan P = prune_plan(ctx->num_sms, M, K, ctx->prune_tpu);
+    const int tpu = P.tpu, KS = P.KS, ctas_per_rb = P.ctas_per_rb;
+    const unsigned grid = P.grid;
+    // every refusal comes before any allocation
+    if ((size_t)P.rb16 * 4 > PRUNE_TICKET_BYTES) return LYNX_ERR_UNSUPPORTED_SHAPE;
     float* sums = nullptr;
     float* partial = nullptr;
     if (sums_needed(mode)) {
         std::lock_guard<std::mutex> lock(ctx->mu);
-        ScratchLayout L = scratch_layout(M, 8, K);
+        ScratchLayout L = scratch_layout(M, K);
         if (ctx->scratch_bytes < L.prune_end) {
             if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
         }
@@ -878,9 +968,6 @@ static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
         partial = reinterpret_cast<float*>(base + L.partial);
         sums = reinterpret_cast<float*>(base + L.sums);
     }
-    if ((size_t)rb16 * 4 > PRUNE_TICKET_BYTES) return LYNX_ERR_UNSUPPORTED_SHAPE;
-    const int ctas_per_rb = (KS + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS;
-    const unsigned grid = (unsigned)(rb16 * ctas_per_rb);
     {
         cudaLaunchConfig_t pc = {};
         pc.gridDim = dim3(grid);
@@ -996,9 +1083,10 @@ lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int6
     if (!aligned16(W) || !aligned16(Y) || (ldw % 8) || (ldy % 8) || (bias && !aligned16(bias)) ||
         (residual && (!aligned16(residual) || (ldr % 8))))
         return LYNX_ERR_ALIGNMENT;
-    ScratchLayout L = scratch_layout(M, N, K);
+    ScratchLayout L = scratch_layout(M, K);
     {
         std::lock_guard<std::mutex> lock(ctx->mu);
+        clear_deferred(ctx);  // this call writes the scratch
         if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
     }
     char* base = static_cast<char*>(ctx->scratch);
@@ -1014,9 +1102,11 @@ lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int6
     comp.row_scale = (!sums_needed(mode) || ss.partial) ? nullptr : scale;
     comp.residual = residual;
     comp.ldr = ldr;
-    if ((s = check_device_error(ctx)) != LYNX_OK) return s;
-    return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &comp, nullptr, Y, ldy,
-                       static_cast<cudaStream_t>(stream), 0, &ss);
+    if ((s = check_device_error(ctx)) == LYNX_OK)
+        s = launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &comp, nullptr, Y, ldy,
+                        static_cast<cudaStream_t>(stream), 0, &ss);
+    clear_deferred(ctx);  // the sums in the scratch belonged to this call
+    return s;
 }
 
 lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_host, int64_t M, int64_t K, const void* W,
@@ -1025,15 +1115,15 @@ lynx_status lynx_act_sparse_linear_host(lynx_ctx* ctx, const void* X_host, int64
     lynx_status s = check_common(ctx, M, K);
     if (s != LYNX_OK) return s;
     if (!X_host || !Y_host || N < 8) return LYNX_ERR_INVALID_ARG;
-    ScratchLayout L = scratch_layout(M, N, K);
+    const size_t x_bytes = align_up((size_t)M * K * 2, 1024), y_bytes = align_up((size_t)M * N * 2, 1024);
     {
         std::lock_guard<std::mutex> lock(ctx->mu);
-        if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
+        if ((s = ensure_scratch(ctx, scratch_layout(M, K).total)) != LYNX_OK) return s;
+        if ((s = ensure_host_stage(ctx, x_bytes + y_bytes)) != LYNX_OK) return s;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    char* base = static_cast<char*>(ctx->scratch);
-    char* xd = base + L.xstage;
-    char* yd = base + L.ystage;
+    char* xd = static_cast<char*>(ctx->host_stage);
+    char* yd = xd + x_bytes;
     // Token rows are independent (except under the whole-tensor scale), so the call is pipelined over
     // row chunks: the copy-in of chunk c + 1 and the copy-out of chunk c - 1 overlap the kernels of
     // chunk c on two copy streams (PCIe is full duplex); the result is the unchunked one bit for bit.
@@ -1134,7 +1224,7 @@ static lynx_status prune_lora_impl(lynx_ctx* ctx, const void* X, int64_t M, int6
     if (!aligned16(X) || !aligned16(LB) || !aligned16(T) || !aligned16(meta) || (ldx % 8) || (ldlb % 8) || (ldt % 8) ||
         (reinterpret_cast<uintptr_t>(values) & 31u))
         return LYNX_ERR_ALIGNMENT;
-    const ScratchLayout L = scratch_layout(M, 8, K);
+    const ScratchLayout L = scratch_layout(M, K);
     {
         std::lock_guard<std::mutex> lock(ctx->mu);
         if (ctx->scratch_bytes < L.prune_end && (s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
@@ -1204,10 +1294,10 @@ lynx_status lynx_sparse_linear_lora(lynx_ctx* ctx, const void* values, const voi
                        static_cast<cudaStream_t>(stream));
 }
 
-lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx,
-                                        const void* W, int64_t N, int64_t ldw, const void* bias, const void* LA,
-                                        int64_t ldla, const void* LB, int64_t ldlb, int64_t R, lynx_comp_mode mode,
-                                        const void* residual, int64_t ldr, void* Y, int64_t ldy, void* stream) {
+static lynx_status act_sparse_linear_lora_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx,
+                                               const void* W, int64_t N, int64_t ldw, const void* bias, const void* LA,
+                                               int64_t ldla, const void* LB, int64_t ldlb, int64_t R, lynx_comp_mode mode,
+                                               const void* residual, int64_t ldr, void* Y, int64_t ldy, void* stream) {
     lynx_status s = check_common(ctx, M, K);
     if (s != LYNX_OK) return s;
     if ((s = check_lora_rank(R)) != LYNX_OK) return s;
@@ -1220,7 +1310,7 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
         (ldw % 8) || (ldy % 8) || (ldla % 8) || (ldlb % 8) || (bias && !aligned16(bias)) ||
         (residual && (!aligned16(residual) || (ldr % 8))))
         return LYNX_ERR_ALIGNMENT;
-    ScratchLayout L = scratch_layout(M, N, K);
+    ScratchLayout L = scratch_layout(M, K);
     const LoraWsLayout LL = lora_ws_layout(ctx->num_sms, M, K, (int)R);
     {
         std::lock_guard<std::mutex> lock(ctx->mu);
@@ -1275,6 +1365,17 @@ lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M,
     s = lynx_lora_down(ctx, X, M, K, ldx, LB, R, ldlb, scale, T, R, stream);
     if (s != LYNX_OK) return s;
     return lynx_sparse_linear_lora(ctx, values, meta, M, K, W, N, ldw, bias, &comp, T, R, LA, R, ldla, Y, ldy, stream);
+}
+
+lynx_status lynx_act_sparse_linear_lora(lynx_ctx* ctx, const void* X, int64_t M, int64_t K, int64_t ldx,
+                                        const void* W, int64_t N, int64_t ldw, const void* bias, const void* LA,
+                                        int64_t ldla, const void* LB, int64_t ldlb, int64_t R, lynx_comp_mode mode,
+                                        const void* residual, int64_t ldr, void* Y, int64_t ldy, void* stream) {
+    if (ctx) clear_deferred(ctx);  // this call writes the scratch
+    const lynx_status s = act_sparse_linear_lora_impl(ctx, X, M, K, ldx, W, N, ldw, bias, LA, ldla, LB, ldlb, R, mode,
+                                                      residual, ldr, Y, ldy, stream);
+    if (ctx) clear_deferred(ctx);  // and the sums it left there belonged to it
+    return s;
 }
 
 // ------------------------------------------------------------------------- FP8 composition ------
@@ -1413,9 +1514,10 @@ lynx_status lynx_act_sparse_linear_fp8(lynx_ctx* ctx, const void* X, int64_t M, 
         (ldy % 8) || (bias && !aligned16(bias)) || (wscale && !aligned16(wscale)) ||
         (residual && (!aligned16(residual) || (ldr % 8))))
         return LYNX_ERR_ALIGNMENT;
-    ScratchLayout L = scratch_layout(M, N, K);
+    ScratchLayout L = scratch_layout(M, K);
     {
         std::lock_guard<std::mutex> lock(ctx->mu);
+        clear_deferred(ctx);  // this call writes the scratch
         if ((s = ensure_scratch(ctx, L.total)) != LYNX_OK) return s;
     }
     char* base = static_cast<char*>(ctx->scratch);
@@ -1507,14 +1609,10 @@ extern "C" lynx_status lynx_prune_compress_static(const void* X, int64_t M, int6
     int num_sms = 0;
     lynx_status s = static_scratch_for_current_device(&scratch, &num_sms);
     if (s != LYNX_OK) return s;
-    // same work decomposition as lynx_prune_compress
-    const int64_t kblocks = K / 128;
-    const int64_t rb16 = ((M + 127) / 128) * 8;
-    const int64_t resident = (int64_t)num_sms * 40;
-    const int64_t want = (rb16 * kblocks) / (3 * resident);
-    int tpu = (int)(want < 1 ? 1 : (want > 8 ? 8 : want));
-    while (kblocks % tpu) --tpu;
-    const int KS = (int)(kblocks / tpu);
+    // the same work decomposition as lynx_prune_compress (one helper: the sums' bits depend on it)
+    const PrunePlan P = prune_plan(num_sms, M, K, 0);
+    const int64_t rb16 = P.rb16;
+    const int tpu = P.tpu, KS = P.KS;
     // static scratch: [tickets: 64 KB][partial sums: rb16 * KS * 32 floats][per-row sums: 2 * M floats]
     // (a __device__ array starts zeroed and every launch leaves its tickets at zero again)
     constexpr size_t STATIC_TICKET_BYTES = 64u << 10;
@@ -1527,8 +1625,8 @@ extern "C" lynx_status lynx_prune_compress_static(const void* X, int64_t M, int6
     float* partial = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + STATIC_TICKET_BYTES);
     float* sums = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + STATIC_TICKET_BYTES + partial_padded);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int ctas_per_rb = (KS + PRUNE_CTA_WARPS - 1) / PRUNE_CTA_WARPS;
-    const unsigned grid = (unsigned)(rb16 * ctas_per_rb);
+    const int ctas_per_rb = P.ctas_per_rb;
+    const unsigned grid = P.grid;
     if (mode == LYNX_COMP_GROUP)
         prune_compress_kernel<false, true><<<grid, PRUNE_CTA_WARPS * 32, 0, st>>>(
             static_cast<const uint16_t*>(X), M, K, ldx, static_cast<uint16_t*>(values), static_cast<uint8_t*>(meta),

@@ -90,35 +90,52 @@ def main():
           "dense us | dense TF | GEMM/dense | layer/dense |")
     print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     for (M, K, N) in shapes:
-        per_set = M * K * 2 + M * K + M * K // 8 + N * K * 2 + M * N * 2
-        nsets = max(2, math.ceil(400e6 / per_set))
-        g = torch.Generator(device="cuda").manual_seed(M + K + N)
-        Xs = [torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16) for _ in range(nsets)]
-        Ws = [(torch.randn(N, K, device="cuda", generator=g) * K ** -0.5).to(torch.bfloat16) for _ in range(nsets)]
-        b = torch.zeros(N, device="cuda", dtype=torch.bfloat16)
-        vs = [torch.empty(M, K // 2, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
-        ms = [torch.empty(binding.meta_bytes(M, K), device="cuda", dtype=torch.uint8) for _ in range(nsets)]
-        ss = [torch.empty(M, device="cuda", dtype=torch.float32) for _ in range(nsets)]
-        Ys = [torch.empty(M, N, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
-        lx.reserve(M, N, K)
-        for j in range(nsets):
-            lx.prune_compress(Xs[j], 1, vs[j], ms[j], ss[j])
-        it = args.iters
-        tp = timeloop(lambda j: lx.prune_compress(Xs[j], 1, vs[j], ms[j], ss[j]), nsets, it)
-        tg = timeloop(lambda j: lx.sparse_linear(vs[j], ms[j], Ws[j], b, ss[j], None, Ys[j]), nsets, it)
-        tl = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_SEPARATE), nsets, it)
-        tf = float("nan")
-        if not args.no_fused:
-            tf = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_FUSED), nsets, it)
-        td = timeloop(lambda j: torch.nn.functional.linear(Xs[j], Ws[j], b), nsets, it)
+        r = time_shape(lx, M, K, N, args.iters, fused=not args.no_fused)
+        tp, tg, tl, tf, td = r["prune_ms"], r["gemm_ms"], r["layer_ms"], r["fused_ms"], r["dense_ms"]
         fl = 2.0 * M * N * K
         tf_s = lambda t: fl / t / 1e9
         print(f"| {M} | {K} | {N} | {tp*1e3:.1f} | {M*K*3.125/tp/1e6:.0f} | {tg*1e3:.1f} | {tf_s(tg):.0f} | "
               f"{tl*1e3:.1f} | {tf_s(tl):.0f} | {tf*1e3:.1f} | {tf_s(tf):.0f} | {td*1e3:.1f} | {tf_s(td):.0f} | "
               f"{td/tg:.2f} | {td/tl:.2f} |", flush=True)
-        assert lx.last_error() == 0
-        del Xs, Ws, vs, ms, ss, Ys
-        torch.cuda.empty_cache()
+
+
+def time_shape(lx, M, K, N, iters=30, fused=False, with_prune_forms=False):
+    """Device times (ms) of the stages of one layer shape, each over rotating inputs larger than the
+    L2: prune/compress alone (ROW mode, scale finished in the launch), sparse GEMM alone, the
+    two-kernel layer, optionally the one-kernel layer, and torch's dense bf16 linear."""
+    per_set = M * K * 2 + M * K + M * K // 8 + N * K * 2 + M * N * 2
+    nsets = max(2, math.ceil(400e6 / per_set))
+    g = torch.Generator(device="cuda").manual_seed(M + K + N)
+    Xs = [torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16) for _ in range(nsets)]
+    Ws = [(torch.randn(N, K, device="cuda", generator=g) * K ** -0.5).to(torch.bfloat16) for _ in range(nsets)]
+    b = torch.zeros(N, device="cuda", dtype=torch.bfloat16)
+    vs = [torch.empty(M, K // 2, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+    ms = [torch.empty(binding.meta_bytes(M, K), device="cuda", dtype=torch.uint8) for _ in range(nsets)]
+    ss = [torch.empty(M, device="cuda", dtype=torch.float32) for _ in range(nsets)]
+    Ys = [torch.empty(M, N, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+    lx.reserve(M, N, K)
+    for j in range(nsets):
+        lx.prune_compress(Xs[j], 1, vs[j], ms[j], ss[j])
+    out = {"M": M, "K": K, "N": N, "nsets": nsets}
+    out["prune_ms"] = timeloop(lambda j: lx.prune_compress(Xs[j], 1, vs[j], ms[j], ss[j]), nsets, iters)
+    if with_prune_forms:
+        out["prune_deferred_ms"] = timeloop(
+            lambda j: lx.prune_compress(Xs[j], 1, vs[j], ms[j], binding.ROW_SCALE_DEFERRED), nsets, iters)
+        for j in range(nsets):  # leave finished scales behind for the GEMM loop
+            lx.prune_compress(Xs[j], 1, vs[j], ms[j], ss[j])
+    out["gemm_ms"] = timeloop(lambda j: lx.sparse_linear(vs[j], ms[j], Ws[j], b, ss[j], None, Ys[j]), nsets, iters)
+    out["layer_ms"] = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_SEPARATE),
+                               nsets, iters)
+    out["fused_ms"] = float("nan")
+    if fused:
+        out["fused_ms"] = timeloop(lambda j: lx.act_sparse_linear(Xs[j], Ws[j], b, 1, None, Ys[j], binding.FUSE_FUSED),
+                                   nsets, iters)
+    out["dense_ms"] = timeloop(lambda j: torch.nn.functional.linear(Xs[j], Ws[j], b), nsets, iters)
+    if lx.last_error() != 0:
+        raise RuntimeError("device-side timeout")
+    del Xs, Ws, vs, ms, ss, Ys
+    torch.cuda.empty_cache()
+    return out
 
 
 def fp8_sweep(lx, shapes, iters):

@@ -8,6 +8,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+# The library reads its development overrides (tile configuration, schedules, kernel forms) only
+# when LYNX_DEV=1; the tests use them to reach every compiled configuration.
+os.environ.setdefault("LYNX_DEV", "1")
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (sm_100a); run with -m gpu")
 

@@ -12,6 +12,7 @@ import torch
 
 import oracle
 from paper_2605_26632_b200 import inputs
+from row_sampling import parity_rows, take
 
 pytestmark = pytest.mark.gpu
 
@@ -260,16 +261,19 @@ def test_every_fp8_tile_configuration(cfg, monkeypatch):
 
 @pytest.mark.parametrize("name", ["mlp_down", "attn_qkv", "mlp_up"])
 def test_dit_workloads_full_size_fp8(lx, name):
+    """Weight codes bit-exact.  Y against the oracle on every row and column for mlp_down (the
+    bench's shape); the oracle's FP8 product takes ~90 s for 4096 rows on the host cores, so the
+    two other shapes are compared on 1024 rows: the first and last row of every 128-row block (the
+    rows one CTA owns) plus a seeded remainder, all N columns -- every output tile is touched."""
     wl = inputs.WORKLOADS[name]
     d = inputs.make_workload(wl, with_bias=True)
-    rows = np.sort(np.random.default_rng(wl.seed).choice(wl.M, 16, replace=False)).astype(np.int64)
-    rows[0], rows[-1] = 0, wl.M - 1
+    rows = parity_rows(wl.M, wl.seed) if name == "mlp_down" else parity_rows(wl.M, wl.seed, all_rows_up_to=0, min_rows=1024)
     oq, ows = oracle.quantize_weights_fp8(u16(d["W"]), True)
     ref = oracle.act_sparse_linear_fp8(u16(d["X"]), oq, ows, bias=u16(d["bias"]), comp_mode=1, rows=rows)
     Wq, ws = lx.quantize_weights_fp8(d["W"].cuda(), True)
     assert (Wq.cpu().numpy() == oq).all()
     Y = lx.act_sparse_linear_fp8(d["X"].cuda(), Wq, ws, d["bias"].cuda(), 1)
-    check_y(Y[torch.from_numpy(rows).cuda()], ref["Y"])
+    check_y(take(Y, rows), ref["Y"])
 
 
 def test_fp8_argument_errors(lx):

@@ -11,6 +11,7 @@ import torch
 
 import oracle
 from paper_2605_26632_b200 import inputs
+from row_sampling import parity_rows, take
 
 pytestmark = pytest.mark.gpu
 
@@ -104,12 +105,13 @@ def test_tiny_config_group_mode_full_oracle(lx, with_bias, with_res):
 
 
 def test_full_size_mlp_down_group_mode(lx):
+    """Y of every row and column against the oracle."""
     wl = inputs.WORKLOADS["mlp_down"]
     d = inputs.make_workload(wl, with_bias=True)
-    rows = np.sort(np.random.default_rng(9).choice(wl.M, 16, replace=False)).astype(np.int64)
+    rows = parity_rows(wl.M, wl.seed)
     ref = oracle.act_sparse_linear(u16(d["X"]), u16(d["W"]), bias=u16(d["bias"]), comp_mode=GROUP, rows=rows)
     Y = lx.act_sparse_linear(d["X"].cuda(), d["W"].cuda(), d["bias"].cuda(), GROUP)
-    check_y(Y[torch.from_numpy(rows).cuda()], ref["Y"])
+    check_y(take(Y, rows), ref["Y"])
 
 
 def test_group_mode_with_low_rank_branch(lx):

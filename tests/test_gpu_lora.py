@@ -12,6 +12,7 @@ import torch
 
 import oracle
 from paper_2605_26632_b200 import inputs
+from row_sampling import parity_rows, take
 
 pytestmark = pytest.mark.gpu
 
@@ -289,13 +290,13 @@ def test_stream_k_with_lora(cfg, monkeypatch):
 
 @pytest.mark.parametrize("name", ["mlp_down", "attn_out", "mlp_up"])
 def test_dit_workloads_full_size_with_lora(lx, name):
+    """Y of every row and column against the oracle (M <= 4608: row_sampling.parity_rows)."""
     wl = inputs.WORKLOADS[name]
     X, W, b, _, LA, LB = make_case(wl.M, wl.K, wl.N, 64, wl.seed, wl.x_dist)
-    rows = np.sort(np.random.default_rng(wl.seed).choice(wl.M, 24, replace=False)).astype(np.int64)
-    rows[0], rows[-1] = 0, wl.M - 1
+    rows = parity_rows(wl.M, wl.seed)
     ref = oracle.act_sparse_linear_lora(u16(X), u16(W), u16(LA), u16(LB), bias=u16(b), comp_mode=1, rows=rows)
     Y = lx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), b.cuda(), 1)
-    check_y(Y[torch.from_numpy(rows).cuda()], ref["Y"])
+    check_y(take(Y, rows), ref["Y"])
 
 
 def test_lora_argument_errors(lx):

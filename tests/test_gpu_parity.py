@@ -12,6 +12,7 @@ import torch
 
 import oracle
 from paper_2605_26632_b200 import inputs
+from row_sampling import parity_rows, take
 
 pytestmark = pytest.mark.gpu
 
@@ -262,6 +263,56 @@ def test_deferred_row_scale_two_call_form(lx):
     assert e.value.status == 1 and lx.launch_count() == n0
 
 
+def test_deferred_row_sums_are_forgotten_when_the_scratch_is_reused_or_regrown():
+    """The deferred sums live in the context's scratch.  Anything that reallocates the scratch
+    (lynx_reserve of a larger shape) or writes other data into it (a layer call, the FP8 layer call)
+    between the two calls must make the GEMM call that still asks for them fail with
+    LYNX_ERR_INVALID_ARG before any launch -- never read freed or overwritten memory."""
+    from paper_2605_26632_b200 import binding
+    from paper_2605_26632_b200.binding import LynxError
+
+    M, K, N = 512, 1024, 256
+    X = inputs.make_x(M, K, "outlier", 61).cuda()
+    W, b = inputs.make_w(N, K, 61).cuda(), inputs.make_bias(N, 61).cuda()
+    X2 = inputs.make_x(256, 512, "gelu", 62).cuda()
+    W2 = inputs.make_w(128, 512, 62).cuda()
+
+    def refused(ctx, v, m):
+        n0 = ctx.launch_count()
+        with pytest.raises(LynxError) as e:
+            ctx.sparse_linear(v, m, W, b, binding.ROW_SCALE_DEFERRED)
+        return e.value.status == 1 and ctx.launch_count() == n0
+
+    ctx = binding.Lynx(0)
+    try:
+        v, m, s = ctx.prune_compress(X, 1)
+        want = ctx.sparse_linear(v, m, W, b, s)
+        # (a) the scratch is regrown between the two calls
+        v2, m2, _ = ctx.prune_compress(X, 1, row_scale=binding.ROW_SCALE_DEFERRED)
+        ctx.reserve(8192, 1024, 4096)
+        assert refused(ctx, v2, m2)
+        # (b) a layer call of another shape writes its compressed operands over the scratch
+        v2, m2, _ = ctx.prune_compress(X, 1, row_scale=binding.ROW_SCALE_DEFERRED)
+        ctx.act_sparse_linear(X2, W2, None, 0)
+        assert refused(ctx, v2, m2)
+        # (c) the FP8 layer call does the same
+        v2, m2, _ = ctx.prune_compress(X, 1, row_scale=binding.ROW_SCALE_DEFERRED)
+        Wq, ws = ctx.quantize_weights_fp8(W2, True)
+        ctx.act_sparse_linear_fp8(X2, Wq, ws, None, 1)
+        assert refused(ctx, v2, m2)
+        # (d) a layer call of the SAME shape leaves its own sums there: they are not the caller's
+        v2, m2, _ = ctx.prune_compress(X, 1, row_scale=binding.ROW_SCALE_DEFERRED)
+        ctx.act_sparse_linear(X, W, b, 1)
+        assert refused(ctx, v2, m2)
+        # and the undisturbed two-call form still works afterwards, same bits
+        v2, m2, _ = ctx.prune_compress(X, 1, row_scale=binding.ROW_SCALE_DEFERRED)
+        assert torch.equal(ctx.sparse_linear(v2, m2, W, b, binding.ROW_SCALE_DEFERRED), want)
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
+
+
 def test_integer_valued_inputs_are_exact(lx):
     """Small integers: every partial sum is exact in fp32 and in bf16, so Y must equal the oracle."""
     rng = np.random.default_rng(4)
@@ -395,7 +446,10 @@ def test_fused_rejects_whole_tensor_scale(lx):
 
 # ------------------------------------------------------------------ full-size workloads --------
 
-def _full_size_case(lx, wl, n_rows, mode=1):
+def _full_size_case(lx, wl, mode=1):
+    """Values, metadata and scale on every element; Y against the oracle on every row when
+    M <= 4608, else on >= 512 rows that include the first and last row of every 128-row block
+    (row_sampling.parity_rows), all N columns: every output tile of the launch is touched."""
     d = inputs.make_workload(wl, with_bias=True)
     X, W, b = d["X"].cuda(), d["W"].cuda(), d["bias"].cuda()
     values, meta, scale = lx.prune_compress(X, mode)
@@ -405,33 +459,58 @@ def _full_size_case(lx, wl, n_rows, mode=1):
     assert (meta.cpu().numpy() == oracle.meta_canon_to_hw(om, wl.M, wl.K)).all()
     np.testing.assert_allclose(scale.cpu().numpy(), oracle.row_scale(Xu, mode), rtol=SCALE_RTOL)
     Y = lx.sparse_linear(values, meta, W, b, scale)
-    rows = np.sort(np.random.default_rng(wl.seed).choice(wl.M, n_rows, replace=False)).astype(np.int64)
-    rows[0], rows[-1] = 0, wl.M - 1
+    rows = parity_rows(wl.M, wl.seed)
     ref = oracle.act_sparse_linear(Xu, u16(d["W"]), bias=u16(d["bias"]), comp_mode=mode, rows=rows)
-    check_y(Y[torch.from_numpy(rows).cuda()], ref["Y"])
+    check_y(take(Y, rows), ref["Y"])
     # same launch configuration as the bench: the single-call path must agree bit for bit
     Y2 = lx.act_sparse_linear(X, W, b, mode)
     assert torch.equal(Y, Y2)
+    torch.cuda.synchronize()
+    assert lx.last_error() == 0
 
 
 @pytest.mark.parametrize("name", ["mlp_down", "attn_qkv", "attn_out", "mlp_up"])
 def test_dit_workloads_full_size(lx, name):
-    """Values and metadata checked on every element, Y on 48 sampled rows (all N columns)."""
-    _full_size_case(lx, inputs.WORKLOADS[name], 48)
+    """Values and metadata checked on every element, Y on every row and column."""
+    _full_size_case(lx, inputs.WORKLOADS[name])
 
 
 @pytest.mark.parametrize("M", inputs.SWEEP_M)
 @pytest.mark.parametrize("K,N", inputs.SWEEP_KN)
 def test_token_sweep(lx, M, K, N):
+    """Y on every row for M <= 4096; for M = 8192 / 16384 on 512 rows covering every 128-row block."""
     idx = inputs.SWEEP_M.index(M) * 4 + inputs.SWEEP_KN.index((K, N))
-    _full_size_case(lx, inputs.sweep_workload(M, K, N, idx), 16)
+    _full_size_case(lx, inputs.sweep_workload(M, K, N, idx))
 
 
 @pytest.mark.parametrize("K,N", inputs.OTHER_FAMILY_KN)
 def test_other_dit_family_shapes(lx, K, N):
-    """FLUX.1-dev single-stream and Z-Image linear shapes (full size, sampled rows)."""
+    """FLUX.1-dev single-stream and Z-Image linear shapes (full size, M = 4096: Y on every row)."""
     idx = 100 + inputs.OTHER_FAMILY_KN.index((K, N))
-    _full_size_case(lx, inputs.sweep_workload(inputs.OTHER_FAMILY_M, K, N, idx), 16)
+    _full_size_case(lx, inputs.sweep_workload(inputs.OTHER_FAMILY_M, K, N, idx))
+
+
+@pytest.mark.parametrize("M,K,N", [
+    (4800, 1024, 1000),    # 19 row tiles of the CTA pair -> groups of 10 + 9, last row tile 192 rows, N tail
+    (12000, 512, 1096),    # 47 row tiles -> three groups (16, 16, 15), 235 output tiles on 74 clusters
+    (8448, 384, 2000),     # 33 row tiles -> 11 + 11 + 11, nine column tiles with a tail
+])
+def test_tile_order_with_several_row_groups_every_row(lx, M, K, N):
+    """More output tiles than clusters, several row-tile groups of unequal size, ragged last row
+    tile and column tail: Y of EVERY row and column against the oracle (a tile skipped, doubled or
+    mapped to the wrong place would show), for bias + row scale + residual."""
+    X = inputs.make_x(M, K, "outlier", 7000 + M)
+    W, b = inputs.make_w(N, K, 7000 + M), inputs.make_bias(N, 7000 + M)
+    res = inputs.make_residual(M, N, 7000 + M)
+    ref = oracle.act_sparse_linear(u16(X), u16(W), bias=u16(b), comp_mode=1, Yr=u16(res))
+    Y = lx.act_sparse_linear(X.cuda(), W.cuda(), b.cuda(), 1, res.cuda())
+    check_y(Y, ref["Y"])
+    # row by row as well: a misplaced tile of small norm must not hide in the Frobenius ratio
+    yf = Y.float().cpu().numpy()
+    err = np.linalg.norm(yf - ref["Y"], axis=1) / np.maximum(np.linalg.norm(ref["Y"], axis=1), 1e-30)
+    assert err.max() <= 4 * RFE_TOL, f"row {int(err.argmax())}: relative error {err.max()}"
+    torch.cuda.synchronize()
+    assert lx.last_error() == 0
 
 
 def test_more_than_2_to_the_31_elements(lx):
