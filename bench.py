@@ -14,10 +14,18 @@ GEMM launch (scale + bias epilogue).  Prints ONE JSON line.
   launch in a second loop of the same steps issued as two calls; ``roofline_prune`` for the
   HBM-bound prune/compress kernel.
 * ``cpu_baseline`` the CPU oracle, as it stands, on a bounded sample of rows of the same workload.
+* ``sustained`` the same step, the sparse GEMM alone and the dense linear again in interleaved blocks
+  of >= 0.5 s each (seconds of tensor-core work: the GPU settles at its power-capped clocks), with
+  the clocks seen in each leg (``--no-sustained`` skips it).
+* ``sweep``   every other configuration the metric names (attention projections, mlp.up with the
+  one-kernel variant beside it, the 16 shapes of the token sweep): prune, GEMM, layer and dense
+  linear, a few milliseconds each (``--no-sweep`` skips it).
 * ``--impl reference`` times the CPU oracle only (there is no other reference implementation).
 
-Multi-GPU (``--gpus N`` under torchrun): the path does not shard; every rank runs an independent
-replica on its own GPU and the aggregate is reported ("replicas only", weak scaling).
+Multi-GPU (``--gpus N``): the path does not shard; every rank runs an independent replica on its
+own GPU and the aggregate is reported ("replicas only", weak scaling).  Under torchrun the ranks
+come from the environment; started plainly with ``--gpus N`` (N > 1) the script launches its own N
+ranks through ``torch.distributed.run`` on 127.0.0.1.
 """
 from __future__ import annotations
 
@@ -36,9 +44,18 @@ sys.path.insert(0, ROOT)
 METRIC = "2:4-act linear TFLOP/s (dense-equiv) and speedup vs dense bf16 GEMM, 1xB200"
 UNIT = "TFLOP/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse GEMM kernel on the
-# mlp_down workload, from the ncu capture summarised in profiles/ (None until captured).
-NCU_TRAFFIC_BYTES = {"mlp_down": 274294272}
+
+
+def ncu_traffic_bytes(workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on `workload`,
+    as recorded from its profiler capture in ncu_traffic.json next to the capture summaries (None
+    when no capture of the current kernel is recorded)."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get("sparse_gemm", {}).get(workload)
+    except (OSError, ValueError):
+        return None
 
 
 def parse_args():
@@ -53,6 +70,10 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-lora", action="store_true", help="skip the extra measurement of the layer with the low-rank branch")
     ap.add_argument("--no-fp8", action="store_true", help="skip the extra measurement of the layer on FP8 operands")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the seconds-long interleaved legs")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the other configurations (attention projections, mlp.up, token sweep)")
+    ap.add_argument("--launch-check", action="store_true",
+                    help="only check the multi-rank launch and aggregation on the CPU (gloo): no GPU work")
     return ap.parse_args()
 
 
@@ -220,10 +241,79 @@ def run_reference(args):
     print(json.dumps(out), flush=True)
 
 
+def self_launch(args) -> int:
+    """``python bench.py --gpus N`` without torchrun: start the N ranks ourselves (one process per
+    GPU, rendezvous on 127.0.0.1) and return their exit code."""
+    import socket
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def launch_check(args):
+    """The multi-rank plumbing without a GPU: gloo ranks, the two aggregation helpers, one JSON line."""
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    ms = max_over_ranks(10.0 + 5.0 * rank, world, device="cpu")
+    value = aggregate_tflops(1e12, 10, ms, world)
+    if rank == 0:
+        print(json.dumps({"launch_check": True, "n_gpus": world, "requested_gpus": args.gpus,
+                          "slowest_rank_ms": ms, "aggregate_tflops": value}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def sustained_legs(legs, ms_guess, sampler, block_s=0.5, rounds=4):
+    """Runs the named legs (name -> callable(i)) in interleaved blocks of >= block_s seconds each,
+    `rounds` times round-robin, so that every leg sees the same thermal / power state.  One CUDA-event
+    pair and one synchronisation per block.  -> name -> dict(ms_per_step, blocks, clocks)."""
+    import torch
+
+    stream = torch.cuda.current_stream()
+    out = {name: {"ms": [], "windows": []} for name in legs}
+    for _ in range(rounds):
+        for name, fn in legs.items():
+            n = max(8, int(block_s * 1e3 / max(ms_guess[name], 1e-3)) + 1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            t0 = time.time()
+            e0.record(stream)
+            for i in range(n):
+                fn(i)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            t1 = time.time()
+            out[name]["ms"].append(e0.elapsed_time(e1) / n)
+            out[name]["windows"].append((t0, t1))
+    res = {}
+    for name, d in out.items():
+        rows = [smp for (t0, t1) in d["windows"] for smp in sampler.samples if t0 <= smp[0] <= t1]
+        reasons = sorted({nm for r in rows for bit, nm in ClockSampler.REASONS.items() if r[3] & bit})
+        pw = [r[2] for r in rows if r[2] == r[2]]
+        res[name] = {"ms_per_step": statistics.median(d["ms"]), "ms_per_step_blocks": d["ms"],
+                     "sm_mhz_median": statistics.median(r[1] for r in rows) if rows else None,
+                     "power_w_max": max(pw) if pw else None, "reasons": reasons, "clock_samples": len(rows)}
+    return res
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(self_launch(args))
+    if args.launch_check:
+        launch_check(args)
         return
 
     import torch
@@ -405,6 +495,72 @@ def main():
                "how": "lynx_act_sparse_linear_fp8: single-read quantising prune/compress + kind::f8f6f4 sparse GEMM"}
         del Wqs
 
+    # ---- sustained regime: seconds of back-to-back work, interleaved A/B/C so that all legs see the same
+    # power state; the GPU leaves its burst clocks and settles where the power cap puts it
+    sustained = None
+    if not args.no_sustained:
+        for j in range(NSETS):  # finished row scales for the GEMM-alone leg
+            lx.prune_compress(Xs[j], comp_mode, vals[j], metas[j], scales[j] if comp_mode else None)
+        legs = {
+            "layer": lambda i: step(i),
+            "sparse_gemm": lambda i: lx.sparse_linear(vals[i % NSETS], metas[i % NSETS], Ws[i % NSETS], bias,
+                                                      scales[i % NSETS] if comp_mode else None, None, Ys[i % NSETS]),
+            "dense_bf16": lambda i: torch.nn.functional.linear(Xs[i % NSETS], Ws[i % NSETS], bias),
+        }
+        guess = {"layer": total_ms / args.steps, "sparse_gemm": sum(gemm_ms) / len(gemm_ms), "dense_bf16": dense_ms}
+        sl = sustained_legs(legs, guess, sampler)
+        flops_ = 2.0 * M * N * K
+        for name in sl:
+            sl[name]["tflops"] = flops_ / (sl[name]["ms_per_step"] * 1e-3) / 1e12
+            mhz = sl[name]["sm_mhz_median"]
+            # time x clock: what the leg would cost in SM cycles (shows how much of a slowdown is the clock)
+            sl[name]["mcycles_per_step"] = sl[name]["ms_per_step"] * mhz * 1e-3 if mhz else None
+        sustained = {
+            "how": "each leg in blocks of >= 0.5 s, four rounds interleaved layer / sparse GEMM alone / dense linear, "
+                   "same rotating buffers as the timed loop, CUDA events per block, median block; clocks = NVML samples "
+                   "inside the leg's blocks",
+            "layer": sl["layer"], "sparse_gemm": sl["sparse_gemm"], "dense_bf16": sl["dense_bf16"],
+            "speedup_vs_dense_bf16": sl["dense_bf16"]["ms_per_step"] / sl["layer"]["ms_per_step"],
+            "gemm_frac_of_2x_bf16_tflops_sustained": sl["sparse_gemm"]["tflops"] / (2.0 * peaks["bf16_tflops_sustained"]),
+            "layer_frac_of_2x_bf16_tflops_sustained": sl["layer"]["tflops"] / (2.0 * peaks["bf16_tflops_sustained"]),
+            "dense_frac_of_bf16_tflops_sustained": sl["dense_bf16"]["tflops"] / peaks["bf16_tflops_sustained"],
+        }
+
+    # ---- the other configurations the metric names: attention projections, mlp.up (with the one-kernel
+    # variant beside it), the 16 shapes of the token sweep; a few milliseconds per stage and shape
+    sweep = None
+    if not args.no_sweep and world == 1:
+        from paper_2605_26632_b200 import sweep as sweep_mod
+
+        rows = []
+        named = [("attn_qkv", inputs.WORKLOADS["attn_qkv"]), ("attn_out", inputs.WORKLOADS["attn_out"]),
+                 ("mlp_up", inputs.WORKLOADS["mlp_up"])]
+        shapes = [(nm, w.M, w.K, w.N, w.x_dist) for nm, w in named]
+        for Ms in inputs.SWEEP_M:
+            for (Kk, Nn) in inputs.SWEEP_KN:
+                w = inputs.sweep_workload(Ms, Kk, Nn)
+                shapes.append(("sweep", w.M, w.K, w.N, w.x_dist))
+        for (nm, Ms, Kk, Nn, dist_) in shapes:
+            r = sweep_mod.time_shape(lx, Ms, Kk, Nn, iters=30, fused=(nm == "mlp_up"), x_dist=dist_)
+            fl = 2.0 * Ms * Nn * Kk
+            row = {"config": nm, "M": Ms, "K": Kk, "N": Nn,
+                   "prune_us": r["prune_ms"] * 1e3, "gemm_us": r["gemm_ms"] * 1e3, "layer_us": r["layer_ms"] * 1e3,
+                   "dense_us": r["dense_ms"] * 1e3, "layer_over_dense": r["dense_ms"] / r["layer_ms"],
+                   "gemm_over_dense": r["dense_ms"] / r["gemm_ms"], "layer_tflops": fl / r["layer_ms"] / 1e9,
+                   "gemm_frac": fl / r["gemm_ms"] / 1e9 / (2.0 * peaks["bf16_tflops"]),
+                   "prune_frac_of_hbm": Ms * Kk * 3.125 / r["prune_ms"] / 1e6 / peaks["hbm_gbs"]}
+            if nm == "mlp_up":
+                row["fused_us"] = r["fused_ms"] * 1e3
+                row["fused_over_separate"] = r["layer_ms"] / r["fused_ms"]
+            rows.append(row)
+        sweep = {"how": "per shape: prune/compress alone (ROW mode, scale finished in the launch), sparse GEMM alone, the "
+                        "two-kernel layer, torch's dense bf16 linear; inputs drawn on the device by the workload's recipe, "
+                        "rotating over enough copies to exceed the L2; each stage replayed from a CUDA graph for ~6 ms, "
+                        "median of three replays (burst clocks)",
+                 "rows": rows,
+                 "layer_over_dense_min": min(r["layer_over_dense"] for r in rows),
+                 "shapes_where_layer_beats_dense": sum(1 for r in rows if r["layer_over_dense"] > 1.0), "shapes": len(rows)}
+
     # end to end through the host-buffer entry point: pinned X in, pinned Y out, every step
     e2e = None
     if not args.no_e2e:
@@ -462,11 +618,10 @@ def main():
                            "(lynx_prune_compress + lynx_sparse_linear), right after the timed loop"},
         "roofline": {"bound": "tensor", "kernel": "sparse_gemm_kernel", "achieved": gemm_tf, "peak": sparse_peak,
                      "unit": "TFLOP/s", "frac": gemm_tf / sparse_peak,
-                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
+                     "traffic": ncu_traffic_bytes(wl.name),
                      "peak_kind": f"2 x {'bf16_tflops_sustained' if long_run else 'bf16_tflops (burst)'} of "
                                   f"{peaks['source']} peaks; 2:4 sparse bf16 = 2 x dense bf16 (nominal ratio); "
-                                  "dense-equivalent flops",
-                     "frac_of_sustained_peak": gemm_tf / (2.0 * peaks["bf16_tflops_sustained"])},
+                                  "dense-equivalent flops; the seconds-long regime is under `sustained`"},
         "roofline_prune": {"bound": "hbm", "kernel": "prune_compress_kernel", "achieved": prune_gbs,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": prune_gbs / peaks["hbm_gbs"],
                            "frac_of_8TBs_nominal": prune_gbs / 8000.0, "bytes_per_launch": prune_bytes, "ms_per_launch": prune_loop_ms,
@@ -478,6 +633,8 @@ def main():
                                   "figure is kernels.prune_compress_ms",
                            "peak_kind": f"hbm_gbs ({peaks['source']})"},
         "clocks": clocks,
+        "sustained": sustained,
+        "sweep": sweep,
         "e2e": e2e,
         "lora": lora,
         "fp8": fp8,

@@ -332,6 +332,19 @@ LYNX_API lynx_status lynx_meta_to_canonical(lynx_ctx* ctx, const void* meta, int
 LYNX_API lynx_status lynx_decompress(lynx_ctx* ctx, const void* values, const void* meta, int64_t M,
                                      int64_t K, void* Xmasked, void* stream);
 
+/* Host-only views of how the sparse GEMM would be run (nothing is launched, no device is needed):
+ * lynx_gemm_plan returns 1 when, for an (M, N, K) product on a GPU with num_sms SMs, the kernel
+ * that runs two 256-row tiles per W stage is chosen (its number of 512-row items and of CTA pairs
+ * in *doubles / *clusters), 0 when the single-tile kernel is, -1 on bad arguments.
+ * lynx_gemm_schedule_items lists the work items of CTA pair `cluster` for `tiles_m` x `tiles_n`
+ * tiles of 256 x 240 over `clusters` pairs with `doubles` 512-row items: items[4i..4i+3] = first
+ * row tile, column tile, row tiles (1 or 2), ordinal among the pair's single-tile items; returns
+ * the item count (only the first `capacity` are written) or -1. */
+LYNX_API int lynx_gemm_plan(int num_sms, int64_t M, int64_t N, int64_t K, int lora_steps, int* doubles,
+                            int* clusters);
+LYNX_API int lynx_gemm_schedule_items(int tiles_m, int tiles_n, int clusters, int doubles, int cluster,
+                                      int* items, int capacity);
+
 /* Number of kernels the library launched on this context since creation (for accounting). */
 LYNX_API int64_t lynx_launch_count(lynx_ctx* ctx);
 

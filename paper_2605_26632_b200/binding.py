@@ -24,7 +24,7 @@ EXPORTS = [
     "lynx_meta_to_canonical", "lynx_decompress", "lynx_launch_count", "lynx_prune_compress_static",
     "lynx_reserve_lora", "lynx_lora_down", "lynx_prune_compress_lora", "lynx_sparse_linear_lora", "lynx_act_sparse_linear_lora",
     "lynx_quantize_weights_fp8", "lynx_prune_compress_fp8", "lynx_sparse_linear_fp8",
-    "lynx_act_sparse_linear_fp8",
+    "lynx_act_sparse_linear_fp8", "lynx_gemm_plan", "lynx_gemm_schedule_items",
 ]
 
 
@@ -100,6 +100,8 @@ def load_library() -> ctypes.CDLL:
                                            i64, vp]
     lib.lynx_act_sparse_linear_fp8.argtypes = [vp, vp, i64, i64, i64, vp, vp, i64, i64, vp, vp, i32, vp, i64, vp,
                                                i64, vp]
+    lib.lynx_gemm_plan.argtypes = [i32, i64, i64, i64, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.lynx_gemm_schedule_items.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(i32), i32]
     lib.lynx_launch_count.argtypes = [vp]
     lib.lynx_launch_count.restype = i64
     _lib = lib
@@ -116,6 +118,25 @@ def values_bytes(M: int, K: int) -> int:
 
 def meta_bytes(M: int, K: int) -> int:
     return int(load_library().lynx_meta_bytes(M, K))
+
+
+def gemm_plan(num_sms: int, M: int, N: int, K: int, lora_steps: int = 0):
+    """-> (uses_two_row_tile_kernel, doubles, clusters): host-only view of the GEMM's plan."""
+    d, c = ctypes.c_int(0), ctypes.c_int(0)
+    r = load_library().lynx_gemm_plan(num_sms, M, N, K, lora_steps, ctypes.byref(d), ctypes.byref(c))
+    if r < 0:
+        raise ValueError("lynx_gemm_plan: bad arguments")
+    return bool(r), d.value, c.value
+
+
+def gemm_schedule_items(tiles_m: int, tiles_n: int, clusters: int, doubles: int, cluster: int):
+    """-> list of (first row tile, column tile, row tiles, ordinal) of one CTA pair (host only)."""
+    cap = tiles_m * tiles_n + 1
+    buf = (ctypes.c_int * (4 * cap))()
+    n = load_library().lynx_gemm_schedule_items(tiles_m, tiles_n, clusters, doubles, cluster, buf, cap)
+    if n < 0:
+        raise ValueError("lynx_gemm_schedule_items: bad arguments")
+    return [tuple(buf[4 * i:4 * i + 4]) for i in range(n)]
 
 
 def _ptr(t: Optional[torch.Tensor]):

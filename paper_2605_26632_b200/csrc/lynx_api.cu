@@ -12,6 +12,7 @@
 
 #include "prune_compress.cuh"
 #include "sparse_gemm.cuh"
+#include "sparse_gemm_rt2.cuh"
 #include "fused_linear.cuh"
 #include "lora_down.cuh"
 #include "fp8_path.cuh"
@@ -56,6 +57,8 @@ struct lynx_ctx {
     int gemm_group_m = 16;    // row tiles per group of the GEMM's tile order (LYNX_GEMM_GROUP_M; 0 = one group)
     int pl_force_splits = 0;  // development override: cluster size of the prune + down-projection kernel
     int splitk_force = 1;     // in-cluster split-K of the GEMM for launches with few tiles: 1 = cost model, 0 = off, 2..4 forced
+    int rt2 = -1;             // two-row-tile GEMM kernel: -1 = cost model, 0 = never, 1 = whenever it applies
+    int rt2_doubles = -1;     // development override: number of 512-row items of its schedule
     int prune_finalize = 0;   // row-scale finalize of the stand-alone prune call: 0 = per shape, 1 = in-kernel ticket, 2 = own launch
     // encoded tensor maps of recent launches, keyed by everything that went into the encoding
     // (a layer called again on the same buffers skips cuTensorMapEncodeTiled)
@@ -419,13 +422,126 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     return LYNX_OK;
 }
 
+// ------------------------------------------------------- two-row-tile GEMM kernel (sparse_gemm_rt2) -----
+
+using Rt2Cfg = Gemm2Cfg<240, 3>;
+
+// Modelled time (us) of the slowest cluster for a schedule with D doubles.  Per-K-block times are
+// measured B200 figures: 0.69 us for a 512 x 240 stage (66 KB in flight per CTA and stage, three
+// stages) against 0.465 us for a 256 x 240 stage of sparse_gemm_kernel (0.49 us here); a double's
+// epilogue is exposed (the accumulators are not double-buffered: ~6 us per double including the
+// refill of the ring), a single's hides behind the next single; the switch between the two rings
+// costs a pipeline fill.  Within each class of clusters the one at the first position carries the
+// most singles, so two clusters decide the maximum.
+constexpr double RT2_T1 = 0.49, RT2_T2 = 0.69, RT2_E1 = 0.8, RT2_E2 = 6.0, RT2_SWITCH = 2.0;
+double rt2_makespan(const PairSchedule& sc, double kb) {
+    double worst = 0.0;
+    const int probe[2] = {sc.b % sc.C, 0};  // position 0 (first light cluster), position L (first heavy one)
+    for (int i = 0; i < 2; ++i) {
+        const int c = probe[i];
+        const int nd = sc.num_doubles(c), ns = sc.num_singles(c);
+        const double t = nd * (kb * RT2_T2 + RT2_E2) + ns * (kb * RT2_T1 + RT2_E1) + ((nd && ns) ? RT2_SWITCH : 0.0);
+        if (t > worst) worst = t;
+    }
+    return worst;
+}
+
+struct Rt2Plan {
+    int doubles, clusters;
+    double t_us;
+};
+Rt2Plan rt2_plan(int num_sms, int64_t M, int64_t N, int64_t K, int lora_steps, int force_doubles) {
+    const int tiles_m = (int)((M + 255) / 256), tiles_n = (int)((N + Rt2Cfg::BN - 1) / Rt2Cfg::BN);
+    const int pairs = num_sms / 2;
+    const double kb = (double)(K / 128) + lora_steps;
+    const int dmax = (tiles_m / 2) * tiles_n;
+    Rt2Plan best{0, 1, 1e30};
+    auto consider = [&](int D) {
+        if (D < 0 || D > dmax) return;
+        const int items = tiles_m * tiles_n - D;
+        const int C = items < pairs ? items : pairs;
+        PairSchedule sc;
+        sc.init(tiles_m, tiles_n, C, D, 8);
+        const double t = rt2_makespan(sc, kb);
+        if (t < best.t_us) best = Rt2Plan{D, C, t};
+    };
+    if (force_doubles >= 0) {
+        consider(force_doubles > dmax ? dmax : force_doubles);
+        return best;
+    }
+    // candidates: every cluster the same number of doubles (multiples of the cluster count), all
+    // slots as doubles, and the neighbours that leave the light clusters exactly one single more
+    consider(dmax);
+    for (int a = 0; a * pairs <= dmax; ++a) consider(a * pairs);
+    return best;
+}
+
+template <bool LORA>
+lynx_status launch_gemm_rt2(lynx_ctx* ctx, const Rt2Plan& plan, const void* values, const void* meta, int64_t M,
+                            int64_t K, const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
+                            const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st, const ScaleSrc* ss) {
+    using Cfg = Rt2Cfg;
+    CUtensorMap ta, tb, te, ty, tt, tla;
+    const uint64_t rb = (uint64_t)((M + 127) / 128), kblocks = (uint64_t)(K / 128);
+    if (!make_tmap_2d(ctx, &ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, values, (uint64_t)M, (uint64_t)(K / 2),
+                      (uint64_t)K, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(ctx, &tb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)N, (uint64_t)K, (uint64_t)ldw * 2, 64,
+                      Cfg::BN_CTA, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(ctx, &te, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, meta, rb * kblocks * 2, 256, 1024, 256, 2,
+                      CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_tmap_2d(ctx, &ty, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, (uint64_t)M, (uint64_t)N, (uint64_t)ldy * 2, Cfg::CH,
+                      32, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return LYNX_ERR_CUDA;
+    if (LORA) {
+        if (!make_tmap_2d(ctx, &tt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->T, (uint64_t)M, (uint64_t)lora->R,
+                          (uint64_t)lora->ldt * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap_2d(ctx, &tla, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lora->LA, (uint64_t)N, (uint64_t)lora->R,
+                          (uint64_t)lora->ldla * 2, 64, Cfg::BN_CTA, CU_TENSOR_MAP_SWIZZLE_128B))
+            return LYNX_ERR_CUDA;
+    } else {
+        tt = ta;  // never read: lora_steps = 0
+        tla = tb;
+    }
+    Gemm2Params p;
+    p.M = M; p.N = N; p.K = K;
+    p.row_scale = comp ? comp->row_scale : nullptr;
+    p.scale_partial = ss ? ss->partial : nullptr;
+    p.scale_ks = ss ? ss->ks : 0;
+    p.bias = static_cast<const uint16_t*>(bias);
+    p.residual = comp ? static_cast<const uint16_t*>(comp->residual) : nullptr;
+    p.ldr = comp ? comp->ldr : 0;
+    p.dev_error = ctx->err_dev;
+    p.sched.init((int)((M + 255) / 256), (int)((N + Cfg::BN - 1) / Cfg::BN), plan.clusters, plan.doubles, 8);
+    p.lora_steps = LORA ? lora->R / 64 : 0;
+    auto kern = sparse_gemm_rt2_kernel<Cfg, LORA>;
+    static bool attr_set[MAX_CTX_DEVICES] = {};  // per instantiation
+    if (lynx_status as = allow_dynamic_smem(kern, Cfg::SMEM_BYTES, ctx->device, attr_set); as != LYNX_OK) return as;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(plan.clusters * 2));
+    cfg.blockDim = dim3(Cfg::THREADS);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = ctx->pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, kern, ta, tb, te, ty, tt, tla, p) != cudaSuccess) return LYNX_ERR_CUDA;
+    ctx->launches++;
+    return LYNX_OK;
+}
+
 // Tile configuration for (M, N, K): the development override, else the smallest modelled time.
 // CTA-pair tiles 256 x {256, 240, 192, 128}.  A sparse MMA takes the same time whatever its N
 // (up to 256), so wide tiles win; 240 is the widest that still double-buffers the accumulator.
 // Model: rounds of tiles over the CTA pairs x (K blocks x measured time per K block + exposed
 // epilogue).  Per-K-block times (us) are measured B200 figures for each tile shape; the 256-wide
 // tile has one accumulator buffer, so its epilogue is not hidden.
-int pick_gemm_cfg_model(int num_sms, int64_t M, int64_t N, int64_t K, int lora_steps) {
+int pick_gemm_cfg_model(int num_sms, int64_t M, int64_t N, int64_t K, int lora_steps, double* t_us = nullptr) {
     const int pairs = num_sms / 2;
     const double kb = (double)(K / 128) + lora_steps;
     struct { int id, bn; double t_kb, epi; } cand[4] = {
@@ -438,7 +554,13 @@ int pick_gemm_cfg_model(int num_sms, int64_t M, int64_t N, int64_t K, int lora_s
         const double t = rounds * (kb * c.t_kb + c.epi);
         if (t < best) { best = t; cfg = c.id; }
     }
+    if (t_us) *t_us = best;
     return cfg;
+}
+double gemm_model_time(int num_sms, int64_t M, int64_t N, int64_t K, int lora_steps) {
+    double t = 0.0;
+    pick_gemm_cfg_model(num_sms, M, N, K, lora_steps, &t);
+    return t;
 }
 int pick_gemm_cfg(const lynx_ctx* ctx, int64_t M, int64_t N, int64_t K, int lora_steps) {
     if (ctx->gemm_cfg != 0) return ctx->gemm_cfg;
@@ -450,7 +572,15 @@ bool cfg_supports_l0(int cfg) { return cfg >= 1 && cfg <= 7 && cfg != 6; }
 lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K, const void* W,
                         int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp, const LoraArgs* lora, void* Y,
                         int64_t ldy, cudaStream_t st, int cfg = 0, const ScaleSrc* ss = nullptr) {
-    if (cfg == 0) cfg = pick_gemm_cfg(ctx, M, N, K, lora ? lora->R / 64 : 0);
+    const int lora_steps = lora ? lora->R / 64 : 0;
+    if (cfg == 0 && ctx->gemm_cfg == 0 && ctx->rt2 != 0 && !ctx->streamk && !(lora && lora->X) && M > 256) {
+        // the two-row-tile kernel where its schedule is modelled faster than the best plain tile
+        const Rt2Plan plan = rt2_plan(ctx->num_sms, M, N, K, lora_steps, ctx->rt2_doubles);
+        if (ctx->rt2 == 1 || plan.t_us < 0.98 * gemm_model_time(ctx->num_sms, M, N, K, lora_steps))
+            return lora ? launch_gemm_rt2<true>(ctx, plan, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss)
+                        : launch_gemm_rt2<false>(ctx, plan, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss);
+    }
+    if (cfg == 0) cfg = pick_gemm_cfg(ctx, M, N, K, lora_steps);
 #define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss
     switch (cfg) {
         case 1: return launch_gemm_cfg<GemmCfg<128, 1, 4, 1>>(LYNX_GEMM_ARGS);
@@ -854,6 +984,8 @@ lynx_status lynx_create(lynx_ctx** out, int device) {
         geti("LYNX_GEMM_GROUP_M", &ctx->gemm_group_m);    // row tiles per group of the GEMM's tile order
         geti("LYNX_PL_SPLITS", &ctx->pl_force_splits);    // K splits (= cluster size) of the prune + down-projection kernel
         if (geti("LYNX_FP8_RING", &ctx->fp8_ring)) ctx->fp8_ring_forced = 1;  // 0 = one CTA per 16 rows, n = ring with n warps per row
+        geti("LYNX_RT2", &ctx->rt2);                      // two-row-tile GEMM kernel: 0 never, 1 whenever it applies
+        geti("LYNX_RT2_D", &ctx->rt2_doubles);            // and the number of 512-row items of its schedule
         geti("LYNX_SPLITK", &ctx->splitk_force);          // in-cluster split-K of the GEMM: 0 off, 1 model (default), 2..4 forced
         geti("LYNX_PRUNE_FINALIZE", &ctx->prune_finalize);  // row-scale finalize: 0 model, 1 in-kernel ticket, 2 own launch
     }
@@ -945,6 +1077,15 @@ static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
         return LYNX_ERR_INVALID_ARG;
     if (mode != LYNX_COMP_ROW) defer = false;
     if (sums_needed(mode) && !row_scale && !defer) return LYNX_ERR_INVALID_ARG;
+    // ROW mode with the scale wanted from this call: on long rows the prune launch stops at its
+    // partial sums and a small dependent launch finishes the scale (measured 30.8 against 33.3 us
+    // on 4096 x 12288); on short rows the ticket hand-over inside the prune kernel is faster
+    // (12-13 against 16-17 us at K = 3072).  Same additions in the same order either way.
+    bool own_finalize = false;
+    if (mode == LYNX_COMP_ROW && !defer) {
+        own_finalize = ctx->prune_finalize == 2 || (ctx->prune_finalize == 0 && K >= 8192);
+        if (K / 128 < 2) own_finalize = false;  // one K split: the kernel writes the scale directly
+    }
     if (ldx < K) return LYNX_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(values) || !aligned16(meta) || (ldx % 16) != 0 ||
         (reinterpret_cast<uintptr_t>(X) & 31u) || (reinterpret_cast<uintptr_t>(values) & 31u))
@@ -992,8 +1133,15 @@ static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
                                    none_f, none_u, 0, tpu, KS, ctas_per_rb, 0);
         else
             e = cudaLaunchKernelEx(&pc, prune_compress_kernel<true, false>, Xp, M, K, ldx, vp, mp, row_scale, sums, partial,
-                                   ctx->tickets, (int)mode, tpu, KS, ctas_per_rb, defer ? 1 : 0);
+                                   ctx->tickets, (int)mode, tpu, KS, ctas_per_rb, (defer || (own_finalize && KS > 1)) ? 1 : 0);
         if (e != cudaSuccess) return LYNX_ERR_CUDA;
+        if (own_finalize && KS > 1) {
+            pc.gridDim = dim3((unsigned)((M + 255) / 256));
+            pc.blockDim = dim3(256);
+            const float* cpart = partial;
+            if (cudaLaunchKernelEx(&pc, row_scale_finalize_kernel, cpart, M, KS, row_scale) != cudaSuccess) return LYNX_ERR_CUDA;
+            ctx->launches++;
+        }
     }
     ctx->launches++;
     if (mode == LYNX_COMP_TENSOR) {
@@ -1335,7 +1483,7 @@ static lynx_status act_sparse_linear_lora_impl(lynx_ctx* ctx, const void* X, int
         comp2.ldr = ldr;
         LoraArgs lora2{T, R, LA, ldla, (int)R};
         return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &comp2, &lora2, Y, ldy,
-                           static_cast<cudaStream_t>(stream), cfg, &ss2);
+                           static_cast<cudaStream_t>(stream), 0, &ss2);
     }
     const bool groups_fit = (size_t)((M + 255) / 256) * 8 * 4 <= L0_WORDS_BYTES;
     const bool fused = ctx->lora_fuse && R == 64 && cfg_supports_l0(cfg) && !ctx->streamk && groups_fit;
@@ -1555,6 +1703,31 @@ lynx_status lynx_decompress(lynx_ctx* ctx, const void* values, const void* meta,
         static_cast<const uint16_t*>(values), static_cast<const uint8_t*>(meta), M, K, static_cast<uint16_t*>(Xmasked));
     ctx->launches++;
     return cuda_ok(cudaGetLastError());
+}
+
+// Host-only inspection of the two-row-tile GEMM's plan and schedule (no device is touched).
+int lynx_gemm_plan(int num_sms, int64_t M, int64_t N, int64_t K, int lora_steps, int* doubles, int* clusters) {
+    if (num_sms < 2 || M < 1 || N < 8 || K < 128) return -1;
+    const Rt2Plan plan = rt2_plan(num_sms, M, N, K, lora_steps, -1);
+    if (doubles) *doubles = plan.doubles;
+    if (clusters) *clusters = plan.clusters;
+    return (M > 256 && plan.t_us < 0.98 * gemm_model_time(num_sms, M, N, K, lora_steps)) ? 1 : 0;
+}
+
+int lynx_gemm_schedule_items(int tiles_m, int tiles_n, int clusters, int doubles, int cluster, int* items, int capacity) {
+    if (tiles_m < 1 || tiles_n < 1 || clusters < 1 || cluster < 0 || cluster >= clusters) return -1;
+    PairSchedule sc;
+    sc.init(tiles_m, tiles_n, clusters, doubles, 8);
+    const int n = sc.num_items(cluster);
+    for (int i = 0; i < n && i < capacity; ++i) {
+        int tm0, tn, rows, ordinal;
+        sc.item(cluster, i, tm0, tn, rows, ordinal);
+        items[4 * i + 0] = tm0;
+        items[4 * i + 1] = tn;
+        items[4 * i + 2] = rows;
+        items[4 * i + 3] = ordinal;
+    }
+    return n;
 }
 
 }  // extern "C"

@@ -256,6 +256,9 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
     if (tid < 64) lut[tid] = prune_lut_entry(tid & 15, tid >> 4);
     __syncthreads();
     griddep_wait();  // no-op unless launched as a programmatic dependent of the previous kernel
+    // the kernel behind this one (the sparse GEMM of a layer call, the scale finalize) may place its
+    // CTAs and run its prologue -- barriers, tensor memory, descriptor prefetch -- while this grid works
+    griddep_launch_dependents();
 
     // CTA -> 16-row block and its first K unit; the CTAs of a row block are consecutive
     const int64_t rb16 = blockIdx.x / ctas_per_rb;
@@ -365,6 +368,17 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
         if (active) prune_tile_store(last, va, vb, slab, okA, okB);
         if (row_scale != nullptr && ks == 0 && lane < 16 && row0 + lane < M) row_scale[row0 + lane] = 1.0f;
     }
+}
+
+// Row scale from the partial sums of a prune launch that stopped there (`defer`): one thread per
+// row, the additions in the order of the in-kernel finalize (same bits).  Launched right behind
+// the prune kernel as a programmatic dependent; on long rows (K >= 8192) the two launches together
+// are faster than the ticket hand-over inside the prune kernel, on short rows slower.
+__global__ void __launch_bounds__(256)
+row_scale_finalize_kernel(const float* __restrict__ partial, int64_t M, int KS, float* __restrict__ row_scale) {
+    griddep_wait();
+    const int64_t row = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (row < M) row_scale[row] = row_scale_from_partials(partial, row, KS);
 }
 
 // Whole-tensor scale: s = sqrt(sum_m num_m / (sum_m den_m + eps)), written to every row_scale[m].

@@ -213,6 +213,10 @@ __device__ __forceinline__ void fence_proxy_async_global() {
 // attribute may start while its predecessor in the stream is still draining; it must execute this
 // wait before it touches anything the predecessor wrote (or still reads).
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// The other half: a kernel tells the runtime that the next kernel of the stream (if it was launched
+// as a programmatic dependent) may start its CTAs now.  That kernel's griddep_wait still waits for
+// this whole grid to finish and its writes to be visible; only its prologue runs early.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------- cluster --------
 

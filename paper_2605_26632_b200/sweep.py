@@ -99,14 +99,28 @@ def main():
               f"{td/tg:.2f} | {td/tl:.2f} |", flush=True)
 
 
-def time_shape(lx, M, K, N, iters=30, fused=False, with_prune_forms=False):
+def device_x(M, K, x_dist, g):
+    """Activations drawn on the device by the recipe of inputs.make_x (same distributions, other
+    random numbers: these tensors are for timing, the parity tests use the CPU generator)."""
+    x = torch.randn(M, K, device="cuda", generator=g)
+    if x_dist in ("gelu", "gelu_chan"):
+        x = torch.nn.functional.gelu(x)
+        if x_dist == "gelu_chan":
+            x = x * torch.exp(0.5 * torch.randn(K, device="cuda", generator=g))
+    elif x_dist == "outlier":
+        idx = torch.randperm(K, device="cuda", generator=g)[:K // 100]
+        x[:, idx] *= 20.0
+    return x.to(torch.bfloat16)
+
+
+def time_shape(lx, M, K, N, iters=30, fused=False, with_prune_forms=False, x_dist="normal"):
     """Device times (ms) of the stages of one layer shape, each over rotating inputs larger than the
     L2: prune/compress alone (ROW mode, scale finished in the launch), sparse GEMM alone, the
     two-kernel layer, optionally the one-kernel layer, and torch's dense bf16 linear."""
     per_set = M * K * 2 + M * K + M * K // 8 + N * K * 2 + M * N * 2
     nsets = max(2, math.ceil(400e6 / per_set))
     g = torch.Generator(device="cuda").manual_seed(M + K + N)
-    Xs = [torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16) for _ in range(nsets)]
+    Xs = [device_x(M, K, x_dist, g) for _ in range(nsets)]
     Ws = [(torch.randn(N, K, device="cuda", generator=g) * K ** -0.5).to(torch.bfloat16) for _ in range(nsets)]
     b = torch.zeros(N, device="cuda", dtype=torch.bfloat16)
     vs = [torch.empty(M, K // 2, device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]

@@ -268,6 +268,29 @@ def test_every_tile_configuration_with_lora(cfg, R, fuse, monkeypatch):
         ctx.close()
 
 
+@pytest.mark.parametrize("doubles", [-1, 0, 100000])
+@pytest.mark.parametrize("R", [64, 128])
+def test_two_row_tile_gemm_kernel_with_lora(R, doubles, monkeypatch):
+    """The low-rank stages inside the GEMM kernel that runs two row tiles per W stage."""
+    from paper_2605_26632_b200 import binding
+
+    monkeypatch.setenv("LYNX_RT2", "1")
+    monkeypatch.setenv("LYNX_RT2_D", str(doubles))
+    ctx = binding.Lynx(0)
+    try:
+        M, K, N = 1100, 1664, 1096  # 5 row tiles (odd), ragged rows and columns
+        X, W, b, res, LA, LB = make_case(M, K, N, R, 900 + R, with_res=True)
+        ref = oracle.act_sparse_linear_lora(u16(X), u16(W), u16(LA), u16(LB), bias=u16(b), comp_mode=1, Yr=u16(res))
+        Y = ctx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), b.cuda(), 1, res.cuda())
+        check_y(Y, ref["Y"])
+        Y2 = ctx.act_sparse_linear_lora(X.cuda(), W.cuda(), LA.cuda(), LB.cuda(), b.cuda(), 1, res.cuda())
+        assert torch.equal(Y, Y2)
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
+
+
 @pytest.mark.parametrize("cfg", [4, 7])
 def test_stream_k_with_lora(cfg, monkeypatch):
     from paper_2605_26632_b200 import binding

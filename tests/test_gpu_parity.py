@@ -116,6 +116,31 @@ def test_prune_compress_is_deterministic(lx):
         assert torch.equal(s, t)
 
 
+@pytest.mark.parametrize("M,K", [(300, 8192), (200, 384), (1000, 12288)])
+def test_row_scale_finalize_forms_agree_bit_for_bit(M, K, monkeypatch):
+    """The per-row scale is finished either by the last CTA of a row block inside the prune kernel
+    (ticket) or by a small dependent launch over the partial sums (the default for K >= 8192):
+    the same additions in the same order, so the same bits; both within 1e-5 of the oracle."""
+    from paper_2605_26632_b200 import binding
+
+    X = inputs.make_x(M, K, "gelu_chan", 500 + M)
+    want = oracle.row_scale(u16(X), 1)
+    got = []
+    for form in ("1", "2", "0"):
+        monkeypatch.setenv("LYNX_PRUNE_FINALIZE", form)
+        ctx = binding.Lynx(0)
+        try:
+            values, meta, scale = ctx.prune_compress(X.cuda(), 1)
+            check_compressed(ctx, X.cuda(), values, meta, scale, 1)
+            np.testing.assert_allclose(scale.cpu().numpy(), want, rtol=SCALE_RTOL)
+            got.append(scale.clone())
+            torch.cuda.synchronize()
+            assert ctx.last_error() == 0
+        finally:
+            ctx.close()
+    assert torch.equal(got[0], got[1]) and torch.equal(got[0], got[2])
+
+
 # ------------------------------------------------------------------ silicon pins of the layout --
 
 @pytest.mark.parametrize("M,K", [(128, 128), (256, 512), (300, 1024)])
@@ -442,6 +467,47 @@ def test_fused_rejects_whole_tensor_scale(lx):
     with pytest.raises(binding.LynxError) as e:
         lx.act_sparse_linear(X, W, None, 2, None, fuse=binding.FUSE_FUSED)
     assert e.value.status == 2
+
+
+# ------------------------------------------------------------------ two-row-tile GEMM kernel ----
+
+@pytest.mark.parametrize("doubles", [-1, 0, 1, 3, 100000])
+@pytest.mark.parametrize("M,K,N", [
+    (700, 1664, 1096),    # 3 row tiles (odd: the last one only forms single-tile items), ragged rows and columns
+    (1024, 512, 2000),    # 4 x 9 tiles on 74 CTA pairs
+    (4800, 1024, 1000),   # 19 x 5 tiles: more items than CTA pairs, several rounds, last row tile 192 rows
+])
+def test_two_row_tile_gemm_kernel(M, K, N, doubles, monkeypatch):
+    """The GEMM kernel that runs two 256-row tiles per W stage, forced on, for several numbers of
+    512-row items (-1 = the cost model's choice, 0 = single-tile items only, 100000 = as many as
+    fit): Y of every row and column against the oracle with bias + row scale + residual, and bit
+    for bit the single-tile kernel's result (same MMAs in the same order per tile, same epilogue
+    arithmetic)."""
+    from paper_2605_26632_b200 import binding
+
+    X = inputs.make_x(M, K, "outlier", 8100 + M)
+    W, b = inputs.make_w(N, K, 8100 + M), inputs.make_bias(N, 8100 + M)
+    res = inputs.make_residual(M, N, 8100 + M)
+    ref = oracle.act_sparse_linear(u16(X), u16(W), bias=u16(b), comp_mode=1, Yr=u16(res))
+    monkeypatch.setenv("LYNX_RT2", "1")
+    monkeypatch.setenv("LYNX_RT2_D", str(doubles))
+    ctx = binding.Lynx(0)
+    try:
+        Y = ctx.act_sparse_linear(X.cuda(), W.cuda(), b.cuda(), 1, res.cuda())
+        check_y(Y, ref["Y"])
+        v, m, s = ctx.prune_compress(X.cuda(), 1)
+        assert torch.equal(ctx.sparse_linear(v, m, W.cuda(), b.cuda(), s, res.cuda()), Y)
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
+    monkeypatch.setenv("LYNX_RT2", "0")
+    monkeypatch.setenv("LYNX_GEMM_CFG", "7")
+    ctx = binding.Lynx(0)
+    try:
+        assert torch.equal(ctx.act_sparse_linear(X.cuda(), W.cuda(), b.cuda(), 1, res.cuda()), Y)
+    finally:
+        ctx.close()
 
 
 # ------------------------------------------------------------------ full-size workloads --------

@@ -35,6 +35,60 @@ def test_size_helpers():
     assert lib.lynx_workspace_bytes(256, 512, 512) >= 256 * 256 * 2 + 2 * 4 * 2048 + 256 * 4
 
 
+def test_two_row_tile_schedule_covers_every_tile_exactly_once():
+    """Host logic of the GEMM's work distribution: for any number of row tiles, column tiles,
+    CTA pairs and 512-row items, every 256 x 240 tile is computed exactly once, doubles pair the
+    row tiles 2d / 2d + 1, consecutive single-tile items of a pair alternate accumulators, and
+    the pairs' loads differ by at most one item of each kind."""
+    from paper_2605_26632_b200 import binding
+
+    import itertools
+    import random
+
+    rng = random.Random(0)
+    cases = [(16, 13, 74, 74), (16, 13, 74, 0), (16, 13, 74, 104), (17, 13, 74, 80), (3, 5, 74, 5), (3, 5, 4, 2),
+             (1, 7, 74, 0), (64, 13, 74, 300), (19, 5, 74, 45), (47, 5, 74, 115), (2, 1, 74, 1)]
+    cases += [(rng.randint(1, 40), rng.randint(1, 30), rng.randint(1, 74), rng.randint(0, 700)) for _ in range(60)]
+    for tm, tn, pairs, doubles in cases:
+        dmax = (tm // 2) * tn
+        d_eff = min(doubles, dmax)
+        clusters = max(1, min(pairs, tm * tn - d_eff))
+        seen = {}
+        nd, ns = [], []
+        for c in range(clusters):
+            items = binding.gemm_schedule_items(tm, tn, clusters, doubles, c)
+            singles = [it for it in items if it[2] == 1]
+            assert [it[3] for it in singles] == list(range(len(singles)))  # ordinals 0, 1, 2, ...
+            assert all(it[2] == 2 for it in items[:len(items) - len(singles)])  # doubles first
+            for (m0, n, rows, _) in items:
+                assert rows in (1, 2) and 0 <= n < tn
+                if rows == 2:
+                    assert m0 % 2 == 0 and m0 + 1 < tm
+                for r in range(rows):
+                    assert 0 <= m0 + r < tm
+                    seen[(m0 + r, n)] = seen.get((m0 + r, n), 0) + 1
+            nd.append(len(items) - len(singles))
+            ns.append(len(singles))
+        assert len(seen) == tm * tn and set(seen.values()) == {1}, (tm, tn, pairs, doubles)
+        assert sum(nd) == d_eff
+        assert max(nd) - min(nd) <= 1
+        # a pair with one double fewer never has fewer singles than a pair with one double more
+        light = [s_ for d_, s_ in zip(nd, ns) if d_ == min(nd)]
+        heavy = [s_ for d_, s_ in zip(nd, ns) if d_ == max(nd)]
+        if max(nd) != min(nd):
+            assert min(light) >= max(heavy)
+        assert max(light) - min(light) <= 1 and max(heavy) - min(heavy) <= 1
+
+
+def test_gemm_plan_prefers_single_tiles_for_small_problems():
+    from paper_2605_26632_b200 import binding
+
+    use, d, c = binding.gemm_plan(148, 1024, 3072, 3072)
+    assert d == 0 or not use  # 52 tiles on 74 pairs: pairing row tiles would only serialise them
+    use, d, c = binding.gemm_plan(148, 4096, 3072, 12288)
+    assert c == 74 and 0 <= d <= 8 * 13
+
+
 def test_status_strings():
     from paper_2605_26632_b200 import binding
 
@@ -90,3 +144,18 @@ def test_replica_aggregation_two_ranks_gloo(tmp_path):
     outs = [p.communicate(timeout=120)[0] for p in procs]
     for p, o in zip(procs, outs):
         assert p.returncode == 0, o
+
+
+def test_bench_launches_its_own_ranks_when_started_plainly():
+    """``python bench.py --gpus 2`` without torchrun starts two ranks itself (127.0.0.1 rendezvous);
+    checked through the GPU-free launch check: gloo ranks, max-over-ranks and aggregation."""
+    import json
+
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--launch-check"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    line = [l for l in res.stdout.splitlines() if l.startswith("{")][-1]
+    d = json.loads(line)
+    assert d["launch_check"] and d["n_gpus"] == 2 and d["slowest_rank_ms"] == 15.0
+    assert abs(d["aggregate_tflops"] - 1e12 * 10 * 2 / 15e-3 / 1e12) < 1e-6
