@@ -332,6 +332,14 @@ LYNX_API lynx_status lynx_meta_to_canonical(lynx_ctx* ctx, const void* meta, int
 LYNX_API lynx_status lynx_decompress(lynx_ctx* ctx, const void* values, const void* meta, int64_t M,
                                      int64_t K, void* Xmasked, void* stream);
 
+/* Self-test of the device-side time-out path.  Every wait inside the kernels is bounded; when one
+ * runs out the kernel sets the context's error word and returns, and the next call on the context
+ * (or lynx_last_error) reports LYNX_ERR_TIMEOUT.  This entry launches one warp that waits
+ * `limit_us` microseconds (1 .. 100000) on a barrier nobody arrives at, so that exactly this
+ * happens: after synchronising `stream`, the next library call returns LYNX_ERR_TIMEOUT and
+ * lynx_last_error returns LYNX_ERR_TIMEOUT once and clears the word.  Nothing faults. */
+LYNX_API lynx_status lynx_selftest_wait_timeout(lynx_ctx* ctx, int64_t limit_us, void* stream);
+
 /* Host-only views of how the sparse GEMM would be run (nothing is launched, no device is needed):
  * lynx_gemm_plan returns 1 when, for an (M, N, K) product on a GPU with num_sms SMs, the kernel
  * that runs two 256-row tiles per W stage is chosen (its number of 512-row items and of CTA pairs

@@ -24,7 +24,7 @@ EXPORTS = [
     "lynx_meta_to_canonical", "lynx_decompress", "lynx_launch_count", "lynx_prune_compress_static",
     "lynx_reserve_lora", "lynx_lora_down", "lynx_prune_compress_lora", "lynx_sparse_linear_lora", "lynx_act_sparse_linear_lora",
     "lynx_quantize_weights_fp8", "lynx_prune_compress_fp8", "lynx_sparse_linear_fp8",
-    "lynx_act_sparse_linear_fp8", "lynx_gemm_plan", "lynx_gemm_schedule_items",
+    "lynx_act_sparse_linear_fp8", "lynx_gemm_plan", "lynx_gemm_schedule_items", "lynx_selftest_wait_timeout",
 ]
 
 
@@ -102,6 +102,7 @@ def load_library() -> ctypes.CDLL:
                                                i64, vp]
     lib.lynx_gemm_plan.argtypes = [i32, i64, i64, i64, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.lynx_gemm_schedule_items.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(i32), i32]
+    lib.lynx_selftest_wait_timeout.argtypes = [vp, i64, vp]
     lib.lynx_launch_count.argtypes = [vp]
     lib.lynx_launch_count.restype = i64
     _lib = lib
@@ -210,6 +211,10 @@ class Lynx:
 
     def last_error(self) -> int:
         return int(self._lib.lynx_last_error(self._h))
+
+    def selftest_wait_timeout(self, limit_us: int = 1000):
+        """Launches the one-warp kernel whose bounded wait runs out (see lynx_selftest_wait_timeout)."""
+        _check(self._lib.lynx_selftest_wait_timeout(self._h, limit_us, _stream()), "lynx_selftest_wait_timeout")
 
     def launch_count(self) -> int:
         return int(self._lib.lynx_launch_count(self._h))

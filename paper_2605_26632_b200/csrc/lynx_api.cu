@@ -294,10 +294,26 @@ static int gemm_group_rows(const lynx_ctx* ctx, int tiles_m) {
     return (tiles_m + groups - 1) / groups;
 }
 
+// One warp; lane 0 waits on a barrier with no arrivals until the limit expires (see
+// lynx_selftest_wait_timeout).  Nothing faults and nothing waits past the limit.
+__global__ void wait_timeout_probe_kernel(uint32_t* dev_error, uint64_t limit_ns) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t abort_word;
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) (void)mbar_wait_limit(smem_u32(&bar), 0, &abort_word, dev_error, limit_ns);
+    __syncwarp();
+}
+
 template <class Cfg>
 lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K,
                             const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
-                            const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st, const ScaleSrc* ss) {
+                            const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st, const ScaleSrc* ss,
+                            bool layer_call) {
     CUtensorMap ta, tb, te, ty, tt, tla, tx, tlb;
     const uint64_t rb = (uint64_t)((M + 127) / 128), kblocks = (uint64_t)(K / 128);
     if (!make_tmap_2d(ctx, &ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, values, (uint64_t)M, (uint64_t)(K / 2),
@@ -362,6 +378,7 @@ lynx_status launch_gemm_cfg(lynx_ctx* ctx, const void* values, const void* meta,
     p.l0_done_target = 0;
     p.T = nullptr;
     p.ldt = 0;
+    p.w_prefetch = (layer_call && !ctx->streamk) ? 1 : 0;
 
     auto kern = lora ? sparse_gemm_kernel<Cfg, true> : sparse_gemm_kernel<Cfg, false>;
     static bool attr_set[2][MAX_CTX_DEVICES] = {};  // per instantiation (with / without the low-rank code)
@@ -479,7 +496,8 @@ Rt2Plan rt2_plan(int num_sms, int64_t M, int64_t N, int64_t K, int lora_steps, i
 template <bool LORA>
 lynx_status launch_gemm_rt2(lynx_ctx* ctx, const Rt2Plan& plan, const void* values, const void* meta, int64_t M,
                             int64_t K, const void* W, int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp,
-                            const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st, const ScaleSrc* ss) {
+                            const LoraArgs* lora, void* Y, int64_t ldy, cudaStream_t st, const ScaleSrc* ss,
+                            bool layer_call) {
     using Cfg = Rt2Cfg;
     CUtensorMap ta, tb, te, ty, tt, tla;
     const uint64_t rb = (uint64_t)((M + 127) / 128), kblocks = (uint64_t)(K / 128);
@@ -513,6 +531,7 @@ lynx_status launch_gemm_rt2(lynx_ctx* ctx, const Rt2Plan& plan, const void* valu
     p.dev_error = ctx->err_dev;
     p.sched.init((int)((M + 255) / 256), (int)((N + Cfg::BN - 1) / Cfg::BN), plan.clusters, plan.doubles, 8);
     p.lora_steps = LORA ? lora->R / 64 : 0;
+    p.w_prefetch = layer_call ? 1 : 0;
     auto kern = sparse_gemm_rt2_kernel<Cfg, LORA>;
     static bool attr_set[MAX_CTX_DEVICES] = {};  // per instantiation
     if (lynx_status as = allow_dynamic_smem(kern, Cfg::SMEM_BYTES, ctx->device, attr_set); as != LYNX_OK) return as;
@@ -571,17 +590,17 @@ bool cfg_supports_l0(int cfg) { return cfg >= 1 && cfg <= 7 && cfg != 6; }
 
 lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int64_t M, int64_t K, const void* W,
                         int64_t N, int64_t ldw, const void* bias, const lynx_comp* comp, const LoraArgs* lora, void* Y,
-                        int64_t ldy, cudaStream_t st, int cfg = 0, const ScaleSrc* ss = nullptr) {
+                        int64_t ldy, cudaStream_t st, int cfg = 0, const ScaleSrc* ss = nullptr, bool layer_call = false) {
     const int lora_steps = lora ? lora->R / 64 : 0;
     if (cfg == 0 && ctx->gemm_cfg == 0 && ctx->rt2 != 0 && !ctx->streamk && !(lora && lora->X) && M > 256) {
         // the two-row-tile kernel where its schedule is modelled faster than the best plain tile
         const Rt2Plan plan = rt2_plan(ctx->num_sms, M, N, K, lora_steps, ctx->rt2_doubles);
         if (ctx->rt2 == 1 || plan.t_us < 0.98 * gemm_model_time(ctx->num_sms, M, N, K, lora_steps))
-            return lora ? launch_gemm_rt2<true>(ctx, plan, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss)
-                        : launch_gemm_rt2<false>(ctx, plan, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss);
+            return lora ? launch_gemm_rt2<true>(ctx, plan, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss, layer_call)
+                        : launch_gemm_rt2<false>(ctx, plan, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss, layer_call);
     }
     if (cfg == 0) cfg = pick_gemm_cfg(ctx, M, N, K, lora_steps);
-#define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss
+#define LYNX_GEMM_ARGS ctx, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss, layer_call
     switch (cfg) {
         case 1: return launch_gemm_cfg<GemmCfg<128, 1, 4, 1>>(LYNX_GEMM_ARGS);
         case 2: return launch_gemm_cfg<GemmCfg<192, 1, 3, 1>>(LYNX_GEMM_ARGS);
@@ -1136,8 +1155,8 @@ static lynx_status prune_impl(lynx_ctx* ctx, const void* X, int64_t M, int64_t K
                                    ctx->tickets, (int)mode, tpu, KS, ctas_per_rb, (defer || (own_finalize && KS > 1)) ? 1 : 0);
         if (e != cudaSuccess) return LYNX_ERR_CUDA;
         if (own_finalize && KS > 1) {
-            pc.gridDim = dim3((unsigned)((M + 255) / 256));
-            pc.blockDim = dim3(256);
+            pc.gridDim = dim3((unsigned)((M + 15) / 16));
+            pc.blockDim = dim3(128);
             const float* cpart = partial;
             if (cudaLaunchKernelEx(&pc, row_scale_finalize_kernel, cpart, M, KS, row_scale) != cudaSuccess) return LYNX_ERR_CUDA;
             ctx->launches++;
@@ -1252,7 +1271,7 @@ lynx_status lynx_act_sparse_linear(lynx_ctx* ctx, const void* X, int64_t M, int6
     comp.ldr = ldr;
     if ((s = check_device_error(ctx)) == LYNX_OK)
         s = launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &comp, nullptr, Y, ldy,
-                        static_cast<cudaStream_t>(stream), 0, &ss);
+                        static_cast<cudaStream_t>(stream), 0, &ss, true);
     clear_deferred(ctx);  // the sums in the scratch belonged to this call
     return s;
 }
@@ -1483,7 +1502,7 @@ static lynx_status act_sparse_linear_lora_impl(lynx_ctx* ctx, const void* X, int
         comp2.ldr = ldr;
         LoraArgs lora2{T, R, LA, ldla, (int)R};
         return launch_gemm(ctx, values, meta, M, K, W, N, ldw, bias, &comp2, &lora2, Y, ldy,
-                           static_cast<cudaStream_t>(stream), 0, &ss2);
+                           static_cast<cudaStream_t>(stream), 0, &ss2, true);
     }
     const bool groups_fit = (size_t)((M + 255) / 256) * 8 * 4 <= L0_WORDS_BYTES;
     const bool fused = ctx->lora_fuse && R == 64 && cfg_supports_l0(cfg) && !ctx->streamk && groups_fit;
@@ -1701,6 +1720,16 @@ lynx_status lynx_decompress(lynx_ctx* ctx, const void* values, const void* meta,
     const int64_t n = M * (K / 4);
     decompress_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint16_t*>(values), static_cast<const uint8_t*>(meta), M, K, static_cast<uint16_t*>(Xmasked));
+    ctx->launches++;
+    return cuda_ok(cudaGetLastError());
+}
+
+// Self-test of the bounded-wait protocol: one CTA waits, with the given limit, on an mbarrier
+// nobody ever arrives at; the wait gives up, raises the CTA's abort word and the context's error
+// word exactly as a kernel of the path would, and the kernel returns normally.
+lynx_status lynx_selftest_wait_timeout(lynx_ctx* ctx, int64_t limit_us, void* stream) {
+    if (!ctx || limit_us < 1 || limit_us > 100000) return LYNX_ERR_INVALID_ARG;
+    wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->err_dev, (uint64_t)limit_us * 1000ull);
     ctx->launches++;
     return cuda_ok(cudaGetLastError());
 }

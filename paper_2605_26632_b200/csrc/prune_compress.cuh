@@ -370,15 +370,37 @@ prune_compress_kernel(const uint16_t* __restrict__ X, int64_t M, int64_t K, int6
     }
 }
 
-// Row scale from the partial sums of a prune launch that stopped there (`defer`): one thread per
-// row, the additions in the order of the in-kernel finalize (same bits).  Launched right behind
-// the prune kernel as a programmatic dependent; on long rows (K >= 8192) the two launches together
-// are faster than the ticket hand-over inside the prune kernel, on short rows slower.
-__global__ void __launch_bounds__(256)
+// Row scale from the partial sums of a prune launch that stopped there (`defer`): one CTA of 128
+// threads per 16-row block, thread (row, jl) adds the partial sums j = jl, jl + 8, ... and the eight
+// strided sums of a row are then added in ascending order -- the additions of the in-kernel
+// finalize in the same order (same bits), all loads of a thread in flight at once.  Launched right
+// behind the prune kernel as a programmatic dependent.
+__global__ void __launch_bounds__(128)
 row_scale_finalize_kernel(const float* __restrict__ partial, int64_t M, int KS, float* __restrict__ row_scale) {
+    __shared__ float2 red[8][16];
     griddep_wait();
-    const int64_t row = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (row < M) row_scale[row] = row_scale_from_partials(partial, row, KS);
+    griddep_launch_dependents();
+    const int tid = threadIdx.x, row = tid & 15, jl = tid >> 4;
+    const int64_t rb16 = blockIdx.x, row0 = rb16 * 16;
+    const float2* pp = reinterpret_cast<const float2*>(partial) + rb16 * KS * 16 + row;
+    float num = 0.f, den = 0.f;
+    for (int j = jl; j < KS; j += 8) {
+        const float2 v = __ldcg(pp + j * 16);
+        num += v.x;
+        den += v.y;
+    }
+    red[jl][row] = make_float2(num, den);
+    __syncthreads();
+    if (tid < 16 && row0 + tid < M) {
+        num = 0.f;
+        den = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            num += red[j][tid].x;
+            den += red[j][tid].y;
+        }
+        row_scale[row0 + tid] = sqrtf(num / (den + 1e-8f));
+    }
 }
 
 // Whole-tensor scale: s = sqrt(sum_m num_m / (sum_m den_m + eps)), written to every row_scale[m].

@@ -65,8 +65,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // if the phase did not complete within `WAIT_LIMIT_NS`, or if another role already aborted.
 constexpr uint64_t WAIT_LIMIT_NS = 4ull * 1000 * 1000 * 1000;
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* cta_abort,
-                                          uint32_t* dev_error) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile uint32_t* cta_abort,
+                                                uint32_t* dev_error, uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;
     for (uint32_t it = 1;; ++it) {
@@ -75,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*cta_abort) return false;
             uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) {
+            else if (now - t0 > limit_ns) {
                 *cta_abort = 1;
                 atomicExch(dev_error, (uint32_t)DEV_TIMEOUT);
                 __threadfence_system();
@@ -83,6 +83,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* cta_abort,
+                                          uint32_t* dev_error) {
+    return mbar_wait_limit(bar, parity, cta_abort, dev_error, WAIT_LIMIT_NS);
 }
 
 // Bounded wait for a global-memory word (written with release semantics by another CTA) to reach

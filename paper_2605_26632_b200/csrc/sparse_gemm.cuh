@@ -72,6 +72,10 @@ struct GemmParams {
     uint32_t l0_done_target;  // its value once this launch has published all of its groups
     uint16_t* T;           // [M x 64] bf16, leading dimension ldt
     int64_t ldt;
+    // Layer calls: W is not produced by the kernel in front of this one (the library's own prune
+    // launch), so the W tiles of the first ring stages may be fetched before the wait for that
+    // kernel; the direct GEMM entry points leave this 0 (whatever precedes them might write W).
+    int w_prefetch;
 };
 
 // Work distribution over C persistent clusters.  The first floor(T/C)*C tiles go round-robin,
@@ -314,6 +318,29 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     if constexpr (CG == 2) cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // W tiles of the first stages of the first tile, before the wait for the previous kernel
+    int npre = 0;
+    if (warp == 0 && lane == 0 && p.w_prefetch && num_items > 0 && l0_n == 0) {
+        const WorkItem w = sched.get(cluster_id, 0);
+        int tm, tn;
+        tile_coords(w.tile, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
+        const int n0 = tn * BN + (int)rank * Cfg::BN_CTA;
+        npre = (w.kb1 - w.kb0 < STAGES) ? w.kb1 - w.kb0 : STAGES;
+        const uint32_t full0 = (CG == 2) ? mapa(bar_full, 0) : bar_full;
+        for (int s = 0; s < npre; ++s) {
+            const int kb = w.kb0 + s;
+            const uint32_t b_dst = sB + s * Cfg::B_BYTES;
+            if constexpr (CG == 1) {
+                mbar_arrive_expect_tx(bar_full + 8 * s, Cfg::STAGE_BYTES);
+                tma_load_2d(b_dst, &tmap_b, kb * Cfg::BK, n0, bar_full + 8 * s);
+                tma_load_2d(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + Cfg::B_BOX_X, n0, bar_full + 8 * s);
+            } else {
+                if (leader) mbar_arrive_expect_tx(bar_full + 8 * s, 2 * Cfg::STAGE_BYTES);
+                tma_load_2d_pair(b_dst, &tmap_b, kb * Cfg::BK, n0, full0 + 8 * s);
+                tma_load_2d_pair(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + Cfg::B_BOX_X, n0, full0 + 8 * s);
+            }
+        }
+    }
     // everything above overlapped the previous kernel's tail; its results are needed from here on
     griddep_wait();
 
@@ -377,22 +404,28 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     const uint32_t a_dst = sA + stage * Cfg::A_BYTES;
                     const uint32_t b_dst = sB + stage * Cfg::B_BYTES;
                     const uint32_t e_dst = sE + stage * Cfg::E_BYTES;
+                    // (the W tiles and the byte count of the first npre stages were issued before the wait)
+                    const bool pre = wi == 0 && kb - w.kb0 < npre;
                     if constexpr (CG == 1) {
                         const uint32_t bar = bar_full + 8 * stage;
-                        mbar_arrive_expect_tx(bar, Cfg::STAGE_BYTES);
+                        if (!pre) mbar_arrive_expect_tx(bar, Cfg::STAGE_BYTES);
                         tma_load_2d(a_dst, &tmap_a, kb * Cfg::A_BOX_X, m0, bar);
                         tma_load_2d(e_dst, &tmap_e, 0, E_ROWS * (eblk + kb), bar);
-                        tma_load_2d(b_dst, &tmap_b, kb * Cfg::BK, n0, bar);
-                        tma_load_2d(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + Cfg::B_BOX_X, n0, bar);
+                        if (!pre) {
+                            tma_load_2d(b_dst, &tmap_b, kb * Cfg::BK, n0, bar);
+                            tma_load_2d(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + Cfg::B_BOX_X, n0, bar);
+                        }
                     } else {
                         const uint32_t bar = full0 + 8 * stage;
                         // the leader announces the bytes of both CTAs; the peer's bytes may land
                         // first (the count goes negative for a moment, which is allowed)
-                        if (leader) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * Cfg::STAGE_BYTES);
+                        if (leader && !pre) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * Cfg::STAGE_BYTES);
                         tma_load_2d_pair(a_dst, &tmap_a, kb * Cfg::A_BOX_X, m0, bar);
                         tma_load_2d_pair(e_dst, &tmap_e, 0, E_ROWS * (eblk + kb), bar);
-                        tma_load_2d_pair(b_dst, &tmap_b, kb * Cfg::BK, n0, bar);
-                        tma_load_2d_pair(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + Cfg::B_BOX_X, n0, bar);
+                        if (!pre) {
+                            tma_load_2d_pair(b_dst, &tmap_b, kb * Cfg::BK, n0, bar);
+                            tma_load_2d_pair(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + Cfg::B_BOX_X, n0, bar);
+                        }
                     }
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }

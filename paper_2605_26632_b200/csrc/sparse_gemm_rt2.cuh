@@ -120,6 +120,7 @@ struct Gemm2Params {
     uint32_t* dev_error;
     PairSchedule sched;
     int lora_steps;  // R / 64 extra dense stages per item (0 = no low-rank branch)
+    int w_prefetch;  // layer calls: W tiles of the first stages are fetched before the wait for the prune launch
 };
 
 template <int BN_, int STAGES_>
@@ -219,6 +220,26 @@ sparse_gemm_rt2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // W tiles of the first stages of the first item, before the wait for the previous kernel (W is
+    // not its output in a layer call); the producer below skips them
+    int npre = 0;
+    if (warp == 0 && lane == 0 && p.w_prefetch && num_items > 0) {
+        int tm0, tn, rows, ordinal;
+        sched.item(cluster_id, 0, tm0, tn, rows, ordinal);
+        const bool r1 = rows == 1;
+        const int nst = r1 ? Cfg::STAGES1 : STAGES;
+        npre = kblocks < nst ? kblocks : nst;
+        const uint32_t bfull = r1 ? bar_full1 : bar_full;
+        const uint32_t full0 = mapa(bfull, 0);
+        const int n0 = tn * BN + (int)rank * Cfg::BN_CTA;
+        const uint32_t tx = r1 ? (uint32_t)Cfg::SINGLE_TX : (uint32_t)Cfg::STAGE_BYTES;
+        for (int s = 0; s < npre; ++s) {
+            const uint32_t b_dst = r1 ? sA + Cfg::RING1_B + s * Cfg::B_BYTES : sB + s * Cfg::B_BYTES;
+            if (leader) mbar_arrive_expect_tx(bfull + 8 * s, 2 * tx);
+            tma_load_2d_pair(b_dst, &tmap_b, s * Cfg::BK, n0, full0 + 8 * s);
+            tma_load_2d_pair(b_dst + Cfg::B_HALF_BYTES, &tmap_b, s * Cfg::BK + 64, n0, full0 + 8 * s);
+        }
+    }
     // everything above overlapped the previous kernel's tail; its results are needed from here on
     griddep_wait();
 
@@ -258,12 +279,15 @@ sparse_gemm_rt2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                     const uint32_t e_dst = ring1 ? sA + Cfg::RING1_E + stage * Cfg::E_BYTES : sE + stage * 2 * Cfg::E_BYTES;
                     const uint32_t bar = full0 + 8 * stage;
                     if (kb < kblocks) {
+                        const bool pre = it == 0 && kb < npre;  // W tile and byte count went out before the wait
                         // the leader announces the bytes of both CTAs; the peer's bytes may land first
-                        if (leader) mbar_arrive_expect_tx(bfull + 8 * stage, 2 * tx);
+                        if (leader && !pre) mbar_arrive_expect_tx(bfull + 8 * stage, 2 * tx);
                         tma_load_2d_pair(a_dst, &tmap_a, kb * 64, rb0 * Cfg::BM, bar);
                         tma_load_2d_pair(e_dst, &tmap_e, 0, 2 * (rb0 * kblocks + kb), bar);
-                        tma_load_2d_pair(b_dst, &tmap_b, kb * Cfg::BK, n0, bar);
-                        tma_load_2d_pair(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + 64, n0, bar);
+                        if (!pre) {
+                            tma_load_2d_pair(b_dst, &tmap_b, kb * Cfg::BK, n0, bar);
+                            tma_load_2d_pair(b_dst + Cfg::B_HALF_BYTES, &tmap_b, kb * Cfg::BK + 64, n0, bar);
+                        }
                         if (rows == 2) {
                             tma_load_2d_pair(a_dst + Cfg::A_BYTES, &tmap_a, kb * 64, (rb0 + 2) * Cfg::BM, bar);
                             tma_load_2d_pair(e_dst + Cfg::E_BYTES, &tmap_e, 0, 2 * ((rb0 + 2) * kblocks + kb), bar);

@@ -666,3 +666,33 @@ def test_argument_errors_are_reported_not_launched(lx):
     assert lx._lib.lynx_prune_compress_fp8(lx._h, vp, 0, 256, 256, None, vp, mp, c_void_p(Y.data_ptr()), 0, None) == 1
     assert lx.launch_count() == n0
     assert lx.last_error() == 0
+
+
+def test_device_side_timeout_is_reported_and_cleared():
+    """A bounded wait that runs out (one warp waiting 1 ms on a barrier nobody arrives at: nothing
+    faults, the kernel returns) raises the context's error word: the next call on the context is
+    refused with LYNX_ERR_TIMEOUT before launching, lynx_last_error reports it once and clears it,
+    and the context is fully usable afterwards."""
+    from paper_2605_26632_b200 import binding
+    from paper_2605_26632_b200.binding import LynxError
+
+    ctx = binding.Lynx(0)
+    try:
+        X = inputs.make_x(256, 512, "gelu", 1).cuda()
+        W = inputs.make_w(256, 512, 1).cuda()
+        want = ctx.act_sparse_linear(X, W, None, 1)
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+        ctx.selftest_wait_timeout(1000)
+        torch.cuda.synchronize()
+        n0 = ctx.launch_count()
+        with pytest.raises(LynxError) as e:
+            ctx.act_sparse_linear(X, W, None, 1)
+        assert e.value.status == 6 and ctx.launch_count() == n0
+        assert ctx.last_error() == 6      # reported ...
+        assert ctx.last_error() == 0      # ... once, then cleared
+        assert torch.equal(ctx.act_sparse_linear(X, W, None, 1), want)
+        torch.cuda.synchronize()
+        assert ctx.last_error() == 0
+    finally:
+        ctx.close()
