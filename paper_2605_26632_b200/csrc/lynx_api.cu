@@ -446,11 +446,11 @@ using Rt2Cfg = Gemm2Cfg<240, 3>;
 // Modelled time (us) of the slowest cluster for a schedule with D doubles.  Per-K-block times are
 // measured B200 figures: 0.69 us for a 512 x 240 stage (66 KB in flight per CTA and stage, three
 // stages) against 0.465 us for a 256 x 240 stage of sparse_gemm_kernel (0.49 us here); a double's
-// epilogue is exposed (the accumulators are not double-buffered: ~6 us per double including the
-// refill of the ring), a single's hides behind the next single; the switch between the two rings
+// epilogue is exposed (the accumulators are not double-buffered, including the
+// refill of the ring: ~5 us per double), a single's hides behind the next single; the switch between the two rings
 // costs a pipeline fill.  Within each class of clusters the one at the first position carries the
 // most singles, so two clusters decide the maximum.
-constexpr double RT2_T1 = 0.49, RT2_T2 = 0.69, RT2_E1 = 0.8, RT2_E2 = 6.0, RT2_SWITCH = 2.0;
+constexpr double RT2_T1 = 0.49, RT2_T2 = 0.69, RT2_E1 = 0.8, RT2_E2 = 5.0, RT2_SWITCH = 2.0;
 double rt2_makespan(const PairSchedule& sc, double kb) {
     double worst = 0.0;
     const int probe[2] = {sc.b % sc.C, 0};  // position 0 (first light cluster), position L (first heavy one)
@@ -595,7 +595,7 @@ lynx_status launch_gemm(lynx_ctx* ctx, const void* values, const void* meta, int
     if (cfg == 0 && ctx->gemm_cfg == 0 && ctx->rt2 != 0 && !ctx->streamk && !(lora && lora->X) && M > 256) {
         // the two-row-tile kernel where its schedule is modelled faster than the best plain tile
         const Rt2Plan plan = rt2_plan(ctx->num_sms, M, N, K, lora_steps, ctx->rt2_doubles);
-        if (ctx->rt2 == 1 || plan.t_us < 0.98 * gemm_model_time(ctx->num_sms, M, N, K, lora_steps))
+        if (ctx->rt2 == 1 || plan.t_us < gemm_model_time(ctx->num_sms, M, N, K, lora_steps))
             return lora ? launch_gemm_rt2<true>(ctx, plan, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss, layer_call)
                         : launch_gemm_rt2<false>(ctx, plan, values, meta, M, K, W, N, ldw, bias, comp, lora, Y, ldy, st, ss, layer_call);
     }
@@ -1740,7 +1740,7 @@ int lynx_gemm_plan(int num_sms, int64_t M, int64_t N, int64_t K, int lora_steps,
     const Rt2Plan plan = rt2_plan(num_sms, M, N, K, lora_steps, -1);
     if (doubles) *doubles = plan.doubles;
     if (clusters) *clusters = plan.clusters;
-    return (M > 256 && plan.t_us < 0.98 * gemm_model_time(num_sms, M, N, K, lora_steps)) ? 1 : 0;
+    return (M > 256 && plan.t_us < gemm_model_time(num_sms, M, N, K, lora_steps)) ? 1 : 0;
 }
 
 int lynx_gemm_schedule_items(int tiles_m, int tiles_n, int clusters, int doubles, int cluster, int* items, int capacity) {

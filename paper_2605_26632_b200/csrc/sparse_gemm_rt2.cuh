@@ -148,7 +148,8 @@ struct Gemm2Cfg {
     static constexpr int NUM_BARS = 2 * STAGES + 2 * STAGES1 + 4;
     static constexpr int C_BOX_BYTES = 32 * CH * 2;    // one epilogue warp's staging box: 32 rows x 48 columns
     static constexpr int C_BYTES = EPI_WARPS * C_BOX_BYTES;
-    static constexpr int SMEM_BYTES = 1024 /*align slack*/ + STAGES * STAGE_BYTES + C_BYTES + 256;
+    static constexpr int BIAS_BYTES = BN * 2;          // one epilogue warp's copy of the item's bias values (bf16)
+    static constexpr int SMEM_BYTES = 1024 /*align slack*/ + STAGES * STAGE_BYTES + C_BYTES + EPI_WARPS * BIAS_BYTES + 256;
     static_assert(BN % CH == 0 && BN % 16 == 0 && BN_CTA % 8 == 0, "tile N");
     static_assert(B_HALF_BYTES % 1024 == 0, "swizzle atoms need 1024-byte aligned tiles");
     static_assert(E_COL0 + E_COLS * STAGES <= TMEM_COLS && 4 * STAGES1 <= E_COLS * STAGES, "tensor memory budget");
@@ -172,7 +173,8 @@ sparse_gemm_rt2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     const uint32_t sB = sA + STAGES * 2 * Cfg::A_BYTES;         // [stage] B_BYTES
     const uint32_t sE = sB + STAGES * Cfg::B_BYTES;             // [stage][row tile] E_BYTES
     const uint32_t sC = sE + STAGES * 2 * Cfg::E_BYTES;         // [epilogue warp] C_BOX_BYTES
-    const uint32_t sBar = sC + Cfg::C_BYTES;
+    const uint32_t sBias = sC + Cfg::C_BYTES;                   // [epilogue warp] BIAS_BYTES
+    const uint32_t sBar = sBias + Cfg::EPI_WARPS * Cfg::BIAS_BYTES;
     const uint32_t bar_full = sBar, bar_empty = sBar + 8 * STAGES;
     const uint32_t bar_tfull = sBar + 16 * STAGES, bar_tempty = bar_tfull + 16;
     const uint32_t bar_full1 = bar_tempty + 16, bar_empty1 = bar_full1 + 8 * Cfg::STAGES1;  // single-tile ring
@@ -416,15 +418,17 @@ sparse_gemm_rt2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 if (p.scale_partial != nullptr) s = row_scale_from_partials(p.scale_partial, row, p.scale_ks);
                 else if (p.row_scale != nullptr) s = __ldg(p.row_scale + row);
             }
-            float bl_all[NCH][2];
-#pragma unroll
-            for (int c = 0; c < NCH; ++c)
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int idx = u * 32 + lane, n = tn * BN + c * CH + idx;
-                    bl_all[c][u] = 0.f;
-                    if (idx < CH && n < p.N && p.bias != nullptr) bl_all[c][u] = __uint_as_float((uint32_t)__ldg(p.bias + n) << 16);
-                }
+            // the item's bias values go to this warp's own strip of shared memory (30 lanes x 8 bf16);
+            // the conversion below reads them back as broadcast 16-byte loads (a shuffle per value
+            // made the shuffle unit the bottleneck of the five conversion rounds)
+            const uint32_t sb = sBias + (warp - 2) * Cfg::BIAS_BYTES;
+            if (lane < BN / 8) {
+                const int n = tn * BN + lane * 8;
+                uint4 bq = make_uint4(0u, 0u, 0u, 0u);
+                if (p.bias != nullptr && n < p.N) bq = __ldg(reinterpret_cast<const uint4*>(p.bias + n));
+                sts128(sb + lane * 16, bq.x, bq.y, bq.z, bq.w);
+            }
+            __syncwarp();
             if (!mbar_wait(bar_tfull + 8 * g, uses & 1u, cta_abort, p.dev_error)) break;
             ++uses;
             tc_fence_after();
@@ -448,10 +452,13 @@ sparse_gemm_rt2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                         if (lane == 0) mbar_arrive_cluster(tempty0 + 8 * g);
                     }
 #pragma unroll
-                    for (int e = 0; e < CH / 2; ++e) {
-                        const float b0 = __shfl_sync(0xffffffffu, bl_all[c][(2 * e) >> 5], (2 * e) & 31);
-                        const float b1 = __shfl_sync(0xffffffffu, bl_all[c][(2 * e + 1) >> 5], (2 * e + 1) & 31);
-                        packed[c][e] = pack_bf16x2(fmaf(s, __uint_as_float(v[2 * e]), b0), fmaf(s, __uint_as_float(v[2 * e + 1]), b1));
+                    for (int j = 0; j < CH / 8; ++j) {
+                        uint32_t bq[4];
+                        lds128(sb + c * (CH * 2) + j * 16, bq[0], bq[1], bq[2], bq[3]);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            packed[c][4 * j + e] = pack_bf16x2(fmaf(s, __uint_as_float(v[8 * j + 2 * e]), bf16_lo_f(bq[e])),
+                                                               fmaf(s, __uint_as_float(v[8 * j + 2 * e + 1]), bf16_hi_f(bq[e])));
                     }
                 }
 #pragma unroll
@@ -501,10 +508,14 @@ sparse_gemm_rt2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 for (int j = 0; j < CH / 8; ++j) {  // 8 columns (16 bytes of output) at a time
                     const int n = n0 + j * 8;
                     float bv[8];
+                    {
+                        uint32_t bq[4];
+                        lds128(sb + c * (CH * 2) + j * 16, bq[0], bq[1], bq[2], bq[3]);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const int col = j * 8 + e;
-                        bv[e] = __shfl_sync(0xffffffffu, bl_all[c][col >> 5], col & 31);
+                        for (int e = 0; e < 4; ++e) {
+                            bv[2 * e] = bf16_lo_f(bq[e]);
+                            bv[2 * e + 1] = bf16_hi_f(bq[e]);
+                        }
                     }
                     float r[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                     if (n < p.N && row_ok) {
