@@ -446,9 +446,9 @@ using Rt2Cfg = Gemm2Cfg<240, 3>;
 // Modelled time (us) of the slowest cluster for a schedule with D doubles.  Per-K-block times are
 // measured B200 figures: 0.69 us for a 512 x 240 stage (66 KB in flight per CTA and stage, three
 // stages) against 0.465 us for a 256 x 240 stage of sparse_gemm_kernel (0.49 us here); a double's
-// epilogue is exposed (the accumulators are not double-buffered, including the
-// refill of the ring: ~5 us per double), a single's hides behind the next single; the switch between the two rings
-// costs a pipeline fill.  Within each class of clusters the one at the first position carries the
+// epilogue is exposed (the accumulators are not double-buffered: ~5 us per double including the
+// refill of the ring), a single's hides behind the next single; the switch between the two
+// rings costs a pipeline fill.  Within each class of clusters the one at the first position carries the
 // most singles, so two clusters decide the maximum.
 constexpr double RT2_T1 = 0.49, RT2_T2 = 0.69, RT2_E1 = 0.8, RT2_E2 = 5.0, RT2_SWITCH = 2.0;
 double rt2_makespan(const PairSchedule& sc, double kb) {
