@@ -471,32 +471,35 @@ def test_fused_rejects_whole_tensor_scale(lx):
 
 # ------------------------------------------------------------------ two-row-tile GEMM kernel ----
 
+@pytest.mark.parametrize("with_res", [True, False])
 @pytest.mark.parametrize("doubles", [-1, 0, 1, 3, 100000])
 @pytest.mark.parametrize("M,K,N", [
     (700, 1664, 1096),    # 3 row tiles (odd: the last one only forms single-tile items), ragged rows and columns
     (1024, 512, 2000),    # 4 x 9 tiles on 74 CTA pairs
     (4800, 1024, 1000),   # 19 x 5 tiles: more items than CTA pairs, several rounds, last row tile 192 rows
 ])
-def test_two_row_tile_gemm_kernel(M, K, N, doubles, monkeypatch):
+def test_two_row_tile_gemm_kernel(M, K, N, doubles, with_res, monkeypatch):
     """The GEMM kernel that runs two 256-row tiles per W stage, forced on, for several numbers of
     512-row items (-1 = the cost model's choice, 0 = single-tile items only, 100000 = as many as
     fit): Y of every row and column against the oracle with bias + row scale + residual, and bit
     for bit the single-tile kernel's result (same MMAs in the same order per tile, same epilogue
-    arithmetic)."""
+    arithmetic).  With a residual the epilogue works chunk by chunk; without, it converts the whole
+    accumulator row in registers before the first store (two code paths)."""
     from paper_2605_26632_b200 import binding
 
     X = inputs.make_x(M, K, "outlier", 8100 + M)
     W, b = inputs.make_w(N, K, 8100 + M), inputs.make_bias(N, 8100 + M)
-    res = inputs.make_residual(M, N, 8100 + M)
-    ref = oracle.act_sparse_linear(u16(X), u16(W), bias=u16(b), comp_mode=1, Yr=u16(res))
+    res = inputs.make_residual(M, N, 8100 + M) if with_res else None
+    ref = oracle.act_sparse_linear(u16(X), u16(W), bias=u16(b), comp_mode=1, Yr=None if res is None else u16(res))
+    res = None if res is None else res.cuda()
     monkeypatch.setenv("LYNX_RT2", "1")
     monkeypatch.setenv("LYNX_RT2_D", str(doubles))
     ctx = binding.Lynx(0)
     try:
-        Y = ctx.act_sparse_linear(X.cuda(), W.cuda(), b.cuda(), 1, res.cuda())
+        Y = ctx.act_sparse_linear(X.cuda(), W.cuda(), b.cuda(), 1, res)
         check_y(Y, ref["Y"])
         v, m, s = ctx.prune_compress(X.cuda(), 1)
-        assert torch.equal(ctx.sparse_linear(v, m, W.cuda(), b.cuda(), s, res.cuda()), Y)
+        assert torch.equal(ctx.sparse_linear(v, m, W.cuda(), b.cuda(), s, res), Y)
         torch.cuda.synchronize()
         assert ctx.last_error() == 0
     finally:
@@ -505,7 +508,7 @@ def test_two_row_tile_gemm_kernel(M, K, N, doubles, monkeypatch):
     monkeypatch.setenv("LYNX_GEMM_CFG", "7")
     ctx = binding.Lynx(0)
     try:
-        assert torch.equal(ctx.act_sparse_linear(X.cuda(), W.cuda(), b.cuda(), 1, res.cuda()), Y)
+        assert torch.equal(ctx.act_sparse_linear(X.cuda(), W.cuda(), b.cuda(), 1, res), Y)
     finally:
         ctx.close()
 
