@@ -174,6 +174,19 @@ def aggregate_tflops(flops_per_step: float, steps: int, total_ms: float, world: 
     return flops_per_step * steps * world / (total_ms * 1e-3) / 1e12
 
 
+NSETS = 3  # rotating copies of every per-step buffer
+
+
+def workload_config(wl, comp: str, world: int) -> dict:
+    """The `config` object of the JSON line: the same for our arm and for the reference arm (which
+    times a bounded sample of this workload; the sample is described in its `cpu_baseline`)."""
+    M, K, N = wl.M, wl.K, wl.N
+    return {"workload": wl.name, "M": M, "K": K, "N": N, "comp": comp, "fuse": "separate",
+            "parallelism": "replicas only" if world > 1 else "single gpu",
+            "l2": f"inputs larger than L2: {NSETS} rotating copies of X/W/values/metadata/Y, "
+                  f"{(M*K*2 + N*K*2 + M*K + M*K//8 + M*N*2)/1e6:.0f} MB touched per step"}
+
+
 def oracle_sample_rate(wl, comp_mode, target_seconds=15.0):
     """Times the CPU oracle on a bounded sample of rows of the workload.  -> dict for the JSON."""
     import numpy as np
@@ -233,8 +246,7 @@ def run_reference(args):
     out = {"impl": "reference", "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-           "data": "synthetic", "config": {"workload": wl.name, "M": wl.M, "K": wl.K, "N": wl.N,
-                                           "comp": args.comp, "rows_per_step": rows},
+           "data": "synthetic", "config": workload_config(wl, args.comp, max(1, args.gpus)),
            "cpu_baseline": cpu,
            "e2e": {"value": tflops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
@@ -341,7 +353,6 @@ def main():
     # Device-resident inputs, rotated over NSETS distinct copies so that, together with W, values,
     # metadata and Y (>= 246 MB per step for mlp_down), nothing a step reads is left in the 126 MB L2
     # by the previous step.
-    NSETS = 3
     Xs = [d["X"].cuda() if i == 0 else None for i in range(NSETS)]
     for i in range(1, NSETS):
         Xs[i] = torch.roll(Xs[0], shifts=i * 4, dims=0).contiguous()
@@ -606,10 +617,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl.name, "M": M, "K": K, "N": N, "comp": args.comp, "fuse": "separate",
-                   "parallelism": "replicas only" if world > 1 else "single gpu",
-                   "l2": f"inputs larger than L2: {NSETS} rotating copies of X/W/values/metadata/Y, "
-                         f"{(M*K*2 + N*K*2 + M*K + M*K//8 + M*N*2)/1e6:.0f} MB touched per step"},
+        "config": workload_config(wl, args.comp, world),
         "speedup_vs_dense_bf16": dense_ms / ms_per_step,
         "dense_bf16": {"ms": dense_ms, "tflops": flops / (dense_ms * 1e-3) / 1e12, "impl": "torch F.linear (cuBLASLt)",
                        "sm_mhz": clocks_dense.get("sm_mhz")},
