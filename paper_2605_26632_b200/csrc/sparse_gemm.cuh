@@ -183,7 +183,7 @@ struct L0Schedule {
 // (a 128-byte swizzled row of compressed A is then 256 logical K instead of 128, a 128-byte row of
 // W 128 K instead of 64), the metadata of a stage doubles (two 128 x 128 blocks), and the four MMAs
 // of a stage are kind::f8f6f4 with K = 64 each.
-template <int BN_, int CG_, int STAGES_, int CBUFS_, bool FP8_ = false>
+template <int BN_, int CG_, int STAGES_, int CBUFS_, bool FP8_ = false, int CH_ = 0>
 struct GemmCfg {
     static constexpr int BN = BN_, CG = CG_, STAGES = STAGES_, CBUFS = CBUFS_;
     static constexpr bool FP8 = FP8_;
@@ -201,7 +201,7 @@ struct GemmCfg {
     // epilogue chunk: 64 columns (128-byte swizzled staging rows) when BN allows, else 48 columns
     // (96-byte unswizzled rows) -- BN = 240 is the widest tile that leaves room for two
     // accumulator buffers plus the metadata columns in the 512 columns of tensor memory
-    static constexpr int CH = (BN % 64 == 0) ? 64 : 48;
+    static constexpr int CH = CH_ ? CH_ : ((BN % 64 == 0) ? 64 : 48);  // (CH_: narrower staging boxes where shared memory is short)
     static constexpr int C_BOX_BYTES = 32 * CH * 2;  // one warp's 32 x CH bf16 store box
     static constexpr int C_BYTES = 4 * CBUFS * C_BOX_BYTES;
     static constexpr int ACC_STAGES = (2 * BN + E_COLS * STAGES <= 512) ? 2 : 1;

@@ -241,7 +241,7 @@ def test_three_call_form_equals_unfused_layer_bit_for_bit(monkeypatch):
 
 
 @pytest.mark.parametrize("fuse", [2, 1, 0])
-@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6, 7])
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6, 7, 8])
 @pytest.mark.parametrize("R", [64, 128])
 def test_every_tile_configuration_with_lora(cfg, R, fuse, monkeypatch):
     """fuse = 2 (default): the down projection runs in the prune launch; fuse = 1: inside the GEMM

@@ -190,7 +190,7 @@ def test_tiny_config_full_oracle(lx, mode, with_bias, with_res):
     assert torch.equal(Y, Y2)
 
 
-@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6, 7])
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_every_tile_configuration(cfg, monkeypatch):
     """All compiled tile shapes (one- and two-CTA MMAs, 128/192/240/256 columns) give the same answer."""
     from paper_2605_26632_b200 import binding
