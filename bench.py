@@ -46,15 +46,23 @@ UNIT = "TFLOP/s"
 
 
 
-def ncu_traffic_bytes(workload: str):
-    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on `workload`,
-    as recorded from its profiler capture in ncu_traffic.json next to the capture summaries (None
-    when no capture of the current kernel is recorded)."""
+def ncu_traffic_bytes(wl, num_sms: int):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on this
+    workload, as recorded from its profiler capture in ncu_traffic.json next to the capture
+    summaries.  None when no capture is recorded, or when the library would now run the GEMM
+    differently (other kernel or schedule) than it did when the capture was taken."""
+    from paper_2605_26632_b200 import binding
+
     path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
     try:
         with open(path) as f:
-            return json.load(f).get("sparse_gemm", {}).get(workload)
-    except (OSError, ValueError):
+            rec = json.load(f).get("sparse_gemm", {}).get(wl.name)
+        if not rec:
+            return None
+        use, doubles, clusters = binding.gemm_plan(num_sms, wl.M, wl.N, wl.K)
+        now = {"two_row_tile_kernel": bool(use), "doubles": int(doubles), "clusters": int(clusters)}
+        return int(rec["bytes"]) if rec.get("plan") == now else None
+    except (OSError, ValueError, KeyError):
         return None
 
 
@@ -627,7 +635,7 @@ def main():
                            "(lynx_prune_compress + lynx_sparse_linear), right after the timed loop"},
         "roofline": {"bound": "tensor", "kernel": "sparse_gemm_kernel", "achieved": gemm_tf, "peak": sparse_peak,
                      "unit": "TFLOP/s", "frac": gemm_tf / sparse_peak,
-                     "traffic": ncu_traffic_bytes(wl.name),
+                     "traffic": ncu_traffic_bytes(wl, torch.cuda.get_device_properties(local_rank).multi_processor_count),
                      "peak_kind": f"2 x {'bf16_tflops_sustained' if long_run else 'bf16_tflops (burst)'} of "
                                   f"{peaks['source']} peaks; 2:4 sparse bf16 = 2 x dense bf16 (nominal ratio); "
                                   "dense-equivalent flops; the seconds-long regime is under `sustained`"},
